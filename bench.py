@@ -1,0 +1,411 @@
+#!/usr/bin/env python
+"""Benchmark of the HiLoRe hot path on B200: one step = the starred steps of Algorithm 1 for one
+microbatch of the 1.5B-shaped workload (84 saved units, all assigned L), through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is the algorithmic HBM traffic of a step divided by the
+device-timed step duration (inputs resident in HBM); `e2e` is the same with host buffers, the
+host<->device copies inside the timed region; `roofline` is the codec kernel against the measured
+HBM copy bandwidth; `cpu_baseline` is the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "compress+recover HBM GB/s (coeff tokens/s alongside); fraction of HBM roofline"
+WORKLOAD = "1.5B-shaped: 64 prompts x G=8 x 1024 tokens; microbatch of 8 responses (8192 token rows); " \
+           "28 layers x (1536, 1536, 8960) bf16 units, all L, E4M3FN + fp32 scale per 64"
+P, G_, T, MB_RESP, LAYERS, MODEL = 64, 8, 1024, 8, 28, "1.5B"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ---------------------------------------------------------------- accounting (bytes the method must move)
+def codec_bytes(rows, cols, fmt_scaled=True, with_rms=False):
+    n = rows * cols
+    return 3 * n + (4 * n // 64 if fmt_scaled else 0) + (4 * rows if with_rms else 0)
+
+
+def coeff_bytes(slots, with_ref=False, extras=False):
+    return slots * (13 + (4 if with_ref else 0) + (5 if extras else 0))
+
+
+def exposure_bytes(n_tok, U):
+    return n_tok * (5 + 4 * U)
+
+
+def peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------- clocks during the timed region
+class ClockSampler:
+    FIELDS = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown," \
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown," \
+             "clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([f.strip() for f in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------- the workload on one GPU
+class Workload:
+    """Device-resident state of one data-parallel rank: the rollout batch's log-probabilities and one
+    microbatch pool of activation units (reused across microbatches: 5.5 GB, far larger than L2)."""
+
+    def __init__(self, api, synth, seed: int, device):
+        self.api, self.device = api, device
+        ro = synth.rollout(seed, P, G_, T)
+        self.ro = ro
+        self.n_resp = ro.n_resp
+        self.rewards = torch.from_numpy(ro.rewards).to(device)
+        self.logp_new = torch.from_numpy(ro.logp_new).to(device)
+        self.logp_old = torch.from_numpy(ro.logp_old).to(device)
+        self.mask = torch.from_numpy(ro.mask).to(device)
+        self.n_microbatches = self.n_resp // MB_RESP
+        self.rows = MB_RESP * T
+        self.shapes = synth.layer_unit_shapes(MODEL, self.rows, LAYERS)
+        self.U = len(self.shapes)
+        gen = torch.Generator(device=device)
+        gen.manual_seed(seed)
+        self.x = [synth.activation_unit_device(gen, r, c, device) for r, c in self.shapes]
+        self.codes = [torch.empty((r, c), dtype=torch.uint8, device=device) for r, c in self.shapes]
+        self.scales = [torch.empty((r, c // 64), dtype=torch.float32, device=device) for r, c in self.shapes]
+        self.out = [torch.empty((r, c), dtype=torch.bfloat16, device=device) for r, c in self.shapes]
+        self.rms = torch.empty((self.U, self.rows), dtype=torch.float32, device=device)
+        units = [dict(x=self.x[i], codes=self.codes[i], scales=self.scales[i], out=self.out[i], row_rms=self.rms[i],
+                      rows=r, cols=c, fmt=api.FMT_E4M3FN_BLK, block=64) for i, (r, c) in enumerate(self.shapes)]
+        self.units_dev, self.units_host = api.make_unit_table(units, device)
+        self.avail = torch.full((self.U,), api.ACT_L, dtype=torch.uint8, device=device)   # candidate plan: all L
+        self.action = torch.zeros(self.U, dtype=torch.uint8, device=device)
+        self.recompute = torch.zeros(self.U, dtype=torch.uint8, device=device)
+        self.retained = torch.zeros(self.U, dtype=torch.int64, device=device)
+        self.psi = torch.zeros(self.U, dtype=torch.float32, device=device)
+        self.exposure = torch.zeros(self.U, dtype=torch.float32, device=device)
+        kgen = np.random.default_rng(seed + 1)
+        self.kappa = torch.from_numpy(kgen.uniform(0.5, 2.0, self.U).astype(np.float32)).to(device)
+        self.ebar = torch.full((self.U,), 0.025, dtype=torch.float32, device=device)
+        self.omega = torch.empty((MB_RESP, T), dtype=torch.float32, device=device)
+        self.adv = torch.empty(MB_RESP, dtype=torch.float32, device=device)
+        self.ws_bytes = api.hilore_workspace_bytes(self.U, self.rows)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
+        self.n_valid = ro.n_valid
+        self.elements = sum(r * c for r, c in self.shapes)
+        self.bytes_compress = sum(codec_bytes(r, c, True, True) for r, c in self.shapes)
+        self.bytes_recover = sum(codec_bytes(r, c, True, False) for r, c in self.shapes)
+        self.bytes_coeffs = coeff_bytes(self.rows)
+        self.bytes_exposure = exposure_bytes(self.rows, self.U)
+        self.bytes_step = self.bytes_compress + self.bytes_recover + self.bytes_coeffs + self.bytes_exposure
+        self.launches_per_step = 6
+
+    def step(self, mb: int, ev=None):
+        """One microbatch: capture (compress all L candidates + token RMS), coefficients, exposure,
+        risk + gating, recover.  `ev`: optional dict of event pairs recorded around the launches."""
+        api = self.api
+        sl = slice(mb * MB_RESP, (mb + 1) * MB_RESP)
+        rec = (lambda k, i: ev[k][i].record()) if ev is not None else (lambda k, i: None)
+        inf = float("inf")
+        rec("compress", 0)
+        api.hilore_plan_apply(self.units_dev, self.units_host, self.U, api.PHASE_CAPTURE, None, None, None, 0.0, 0.0,
+                              self.avail, self.action, None, None, None)
+        rec("compress", 1)
+        rec("coeffs", 0)
+        api.hilore_grpo_coeffs(self.rewards, self.n_resp, G_, mb * MB_RESP, MB_RESP, T, self.logp_new[sl],
+                               self.logp_old[sl], None, self.mask[sl], self.n_valid, None, 0.2, 0.0, 1e-6,
+                               self.adv, self.omega, None, None)
+        rec("coeffs", 1)
+        rec("exposure", 0)
+        api.hilore_unit_exposure(self.omega, self.mask[sl], MB_RESP, T, self.rms, self.U, self.rows, 0, 1e-8,
+                                 self.exposure, None, self.ws, self.ws_bytes)
+        rec("exposure", 1)
+        api.hilore_plan_apply(self.units_dev, self.units_host, self.U, api.PHASE_DECIDE, self.exposure, self.kappa,
+                              self.ebar, inf, inf, self.avail, self.action, self.psi, self.recompute, self.retained)
+        rec("recover", 0)
+        api.hilore_plan_apply(self.units_dev, self.units_host, self.U, api.PHASE_RECOVER, None, None, None, 0.0, 0.0,
+                              self.avail, self.action, None, None, None)
+        rec("recover", 1)
+
+
+def coeff_sweep_point(api, synth, device, log2_slots=24, reps=10):
+    """Coefficient kernel alone on 2^24 slots at G = 16, T = 1024 (218 MB of traffic, larger than L2)."""
+    n_resp = (1 << log2_slots) // 1024
+    gen = torch.Generator(device=device)
+    gen.manual_seed(5)
+    lp = torch.randn((n_resp, 1024), generator=gen, device=device) * 0.5 - 1.5
+    lo = lp + torch.randn((n_resp, 1024), generator=gen, device=device) * 0.05
+    mask = torch.ones((n_resp, 1024), dtype=torch.uint8, device=device)
+    rewards = (torch.rand(n_resp, generator=gen, device=device) < 0.5).float()
+    omega = torch.empty_like(lp)
+    run = lambda: api.hilore_grpo_coeffs(rewards, n_resp, 16, 0, n_resp, 1024, lp, lo, None, mask, n_resp * 1024, None,
+                                         0.2, 0.0, 1e-6, None, omega, None, None)
+    for _ in range(3):
+        run()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    slots = n_resp * 1024
+    return {"slots": slots, "ms": ms, "tokens_per_s": slots / ms * 1e3, "gbs": coeff_bytes(slots) / ms / 1e6}
+
+
+# ---------------------------------------------------------------- CPU oracle legs
+def oracle_sample_step(synth_mod, seed=0):
+    """The oracle on a bounded sample of the workload: layer 0's three units of one microbatch
+    (compress with token RMS, recover), the microbatch's coefficients, and the exposure of those units.
+    Returns (seconds, algorithmic bytes of the sample)."""
+    import oracle
+    rng = np.random.default_rng(seed)
+    rows = MB_RESP * T
+    shapes = synth_mod.layer_unit_shapes(MODEL, rows, 1)
+    xs = [synth_mod.activation_unit(rng, r, c) for r, c in shapes]
+    ro = synth_mod.rollout(seed, 8, G_, T)          # a slice of the rollout batch is enough for the sample
+    oracle.lib()
+    t0 = time.perf_counter()
+    rms = []
+    recs = 0
+    for x in xs:
+        codes, scales = oracle.compress(x, oracle.FMT_E4M3FN_BLK, 64)
+        rms.append(oracle.row_rms(x))
+        recs += oracle.recover(codes, scales, oracle.FMT_E4M3FN_BLK, 64).size
+    adv = oracle.group_advantages(ro.rewards, G_)
+    omega, _, _ = oracle.grpo_coeffs(adv[:MB_RESP], ro.logp_new[:MB_RESP], ro.logp_old[:MB_RESP], None,
+                                     ro.mask[:MB_RESP], N_norm=P * G_ * T)
+    E, _ = oracle.unit_exposure(omega, ro.mask[:MB_RESP], np.stack(rms))
+    dt = time.perf_counter() - t0
+    nbytes = sum(codec_bytes(r, c, True, True) + codec_bytes(r, c, True, False) for r, c in shapes) \
+        + coeff_bytes(rows) + exposure_bytes(rows, len(shapes))
+    return dt, nbytes
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2609_33570_b200 import synth
+    times = []
+    nbytes = 0
+    for i in range(args.warmup + args.steps):
+        dt, nbytes = oracle_sample_step(synth, seed=i)
+        if i >= args.warmup:
+            times.append(dt)
+    sec = sum(times) / len(times)
+    val = nbytes / sec / 1e9
+    sample = "layer 0 of one microbatch: units [8192,1536]x2 + [8192,8960], coefficients of 8192 slots, exposure U=3"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16->e4m3fn (fp32 scales, fp64 oracle arithmetic)", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample_per_step": sample},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------- main (our arm)
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    if args.warmup < 3:
+        args.warmup = 3
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    from paper_2609_33570_b200 import api, dist as hdist, synth
+
+    wl = Workload(api, synth, seed=rank, device=device)
+    # batch-wide normaliser N: the one exchange of the path (once per update, outside the microbatch step)
+    local_count = torch.zeros(1, dtype=torch.int64, device=device)
+    api.hilore_mask_count(wl.mask, wl.mask.numel(), local_count)
+    n_global = hdist.global_token_count(local_count) if world > 1 else int(local_count.item())
+    wl.n_valid = n_global
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        wl.step(i % wl.n_microbatches)
+    kinds = ("compress", "coeffs", "exposure", "recover")
+    evs = [{k: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for k in kinds}
+           for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    e0.record()
+    for i in range(args.steps):
+        wl.step((args.warmup + i) % wl.n_microbatches, evs[i])
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    kern_ms = {k: sum(e[k][0].elapsed_time(e[k][1]) for e in evs) / args.steps for k in kinds}
+
+    # end to end: host buffers, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        hx = [torch.empty(x.shape, dtype=x.dtype, pin_memory=True) for x in wl.x]
+        for h, x in zip(hx, wl.x):
+            h.copy_(x)
+        h_ln, h_lo, h_mk = (torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for v in
+                            (wl.logp_new, wl.logp_old, wl.mask))
+        h_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in
+                 (("exposure", wl.exposure), ("psi", wl.psi), ("action", wl.action), ("retained", wl.retained))}
+        h2d = sum(h.numel() * h.element_size() for h in hx) + MB_RESP * T * 9
+        d2h = sum(v.numel() * v.element_size() for v in h_out.values())
+
+        def e2e_step(mb):
+            sl = slice(mb * MB_RESP, (mb + 1) * MB_RESP)
+            for h, x in zip(hx, wl.x):
+                x.copy_(h, non_blocking=True)
+            wl.logp_new[sl].copy_(h_ln[sl], non_blocking=True)
+            wl.logp_old[sl].copy_(h_lo[sl], non_blocking=True)
+            wl.mask[sl].copy_(h_mk[sl], non_blocking=True)
+            wl.step(mb)
+            for k, v in (("exposure", wl.exposure), ("psi", wl.psi), ("action", wl.action), ("retained", wl.retained)):
+                h_out[k].copy_(v, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+
+        e2e_step(0)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            e2e_step(i % wl.n_microbatches)
+        barrier()
+        dt = torch.tensor([time.perf_counter() - t0], dtype=torch.float64, device=device)
+        if world > 1:
+            dist.all_reduce(dt, op=dist.ReduceOp.MAX)
+        e2e_s = float(dt.item()) / args.e2e_steps
+        e2e = {"value": world * wl.bytes_step / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": args.e2e_steps}
+        del hx
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = peak_hbm()
+    codec_ms = (kern_ms["compress"] + kern_ms["recover"]) / 2
+    codec_bytes_per_launch = (wl.bytes_compress + wl.bytes_recover) / 2
+    achieved = codec_bytes_per_launch / codec_ms / 1e6
+    sweep = coeff_sweep_point(api, synth, device)
+    out = {
+        "metric": METRIC, "value": world * wl.bytes_step / ms_step / 1e6, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16->e4m3fn codes (fp32 scales, fp32 coefficients)",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (5.5 GB of units per step)",
+                   "units": wl.U, "elements_per_step": wl.elements, "bytes_per_step": wl.bytes_step,
+                   "parallelism": f"dp{world} (microbatches sharded, no data-path collective)"},
+        "gpu_launches": wl.launches_per_step * args.steps,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "codec_kernel (compress and recover launches averaged)",
+                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_8000_nominal": achieved / 8000.0, "traffic": None},
+        "kernels": {
+            "compress": {"ms": kern_ms["compress"], "gbs": wl.bytes_compress / kern_ms["compress"] / 1e6},
+            "recover": {"ms": kern_ms["recover"], "gbs": wl.bytes_recover / kern_ms["recover"] / 1e6},
+            "coeffs_microbatch": {"ms": kern_ms["coeffs"], "tokens_per_s": wl.rows / kern_ms["coeffs"] * 1e3},
+            "exposure": {"ms": kern_ms["exposure"], "gbs": wl.bytes_exposure / kern_ms["exposure"] / 1e6},
+            "coeffs_2p24": sweep,
+        },
+        "coeff_tokens_per_s": sweep["tokens_per_s"],
+        "e2e": e2e,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        dt, nb = oracle_sample_step(synth)
+        out["cpu_baseline"] = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle", "seconds": dt,
+                               "sample": "layer 0 of one microbatch (3 of the 84 units: [8192,1536]x2 + [8192,8960]), "
+                                         "coefficients of 8192 slots, exposure U=3"}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

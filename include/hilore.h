@@ -1,0 +1,207 @@
+/*
+ * hilore.h -- C ABI of the B200 (sm_100a) hot path of HiLoRe's GRPO actor update.
+ *
+ * Two parts (paper: Algorithm 1, lines "Coefficients", "Exposure", risk score, and the
+ * capture / recovery of L units):
+ *   1. the fused GRPO loss-coefficient pass and its reduction to one update-exposure score
+ *      per recovery unit, available before backward (Prop. 1, Eq. "update-coefficient",
+ *      Eq. "mlp-weighted-exposure");
+ *   2. the low-precision store / recover path for saved bf16 activations
+ *      (Eq. "fp8-roundtrip"), gated by the per-unit H / L / R plan
+ *      (Eq. "available-recovery-actions").
+ *
+ * Conventions for every entry point
+ *   - Returns an int status (HILORE_OK = 0).  Never throws, aborts or traps.
+ *   - Every pointer is a DEVICE pointer owned by the caller, valid until the work enqueued
+ *     by the call has finished, unless its comment says "host".
+ *   - The library allocates nothing and keeps no state between calls (the one exception is
+ *     stated at its declaration).  Work is enqueued on `stream` (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and the call returns without synchronising.
+ *     HILORE_CUDA reports a launch error seen by cudaGetLastError, nothing asynchronous.
+ *   - Tensors are row-major.  bf16 tensors are passed as void* (16-bit patterns).
+ *   - Output buffers must not overlap inputs or each other.
+ *   - Optional pointers say "opt" and may be NULL.
+ */
+#ifndef HILORE_H
+#define HILORE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- status codes ---- */
+enum {
+    HILORE_OK = 0,
+    HILORE_INVALID_ARG = 1, /* NULL where data is required, negative size, unknown enum value          */
+    HILORE_SHAPE = 2,       /* cols % 16 != 0, cols % block != 0, n_resp % G != 0, ld < cols, ...       */
+    HILORE_ALIGN = 3,       /* a pointer or leading dimension misses the alignment stated below       */
+    HILORE_ZERO_NORM = 4,   /* the normaliser N is not positive and no device-side N was given         */
+    HILORE_CUDA = 5,        /* kernel launch failed                                                    */
+    HILORE_WORKSPACE = 6    /* workspace too small; see hilore_workspace_bytes                         */
+};
+
+/* ---- storage formats of the L (compress) action ---- */
+enum {
+    HILORE_FMT_E4M3FN_RAW = 0, /* the paper's codec, Eq. "fp8-roundtrip": unscaled cast to FP8 E4M3FN,
+                                  one byte per element, no scales; values that round above 448 and
+                                  non-finite values become the NaN code, as the cast the paper names does */
+    HILORE_FMT_E4M3FN_BLK = 1, /* E4M3FN payload + one fp32 absmax scale per block of 64 elements of a
+                                  row (the benchmark's block-scaled generalisation; not in the paper)    */
+    HILORE_FMT_INT8_BLK = 2    /* INT8 payload (+-127) + one fp32 absmax scale per block of 64            */
+};
+#define HILORE_BLOCK 64 /* the only block size of the scaled formats */
+
+/* ---- recovery actions; the numeric order is the paper's tie order R, H, L ---- */
+enum { HILORE_ACT_R = 0, HILORE_ACT_H = 1, HILORE_ACT_L = 2 };
+
+/* ---- phases of hilore_plan_apply ---- */
+enum {
+    HILORE_PHASE_DECIDE = 0,  /* risk score, threshold rule, availability -> action / recompute / bytes  */
+    HILORE_PHASE_CAPTURE = 1, /* forward-time capture by candidate plan q: q = L compress (+ token RMS),
+                                 q = H token RMS only (bf16 kept), q = R nothing                          */
+    HILORE_PHASE_ENCODE = 2,  /* post-forward encoding: units with q = H that were assigned L           */
+    HILORE_PHASE_RECOVER = 3  /* backward-time recovery: units with action L are decoded to bf16         */
+};
+
+const char *hilore_status_string(int status);
+/* Version of this ABI (major * 1000 + minor). */
+int hilore_abi_version(void);
+
+/*
+ * N = sum_t m_t, the learner's normaliser (Eq. "grpo-objective": N = sum of the update mask; the
+ * setup section normalises by all valid response tokens of the complete rollout batch).
+ *   mask   [n] u8, 0 or 1.            count  one int64 on the device, overwritten with the sum.
+ * The sum is an integer, so the result does not depend on the order of the additions.
+ */
+int hilore_mask_count(const uint8_t *mask, int64_t n, int64_t *count, void *stream);
+
+/*
+ * Group-relative advantages and per-token update coefficients omega_t = dL/ds_t
+ * (Eq. "grpo-objective", Eq. "update-coefficient", K3 derivative in the proof of Prop. 1):
+ *     A_j     = (R_j - mean_g) / (population_std_g + adv_eps); a group whose rewards are all equal
+ *               has A = +0 exactly (setup section, "GRPO and optimization")
+ *     r_t     = exp(s_t - s_old_t)
+ *     chi_t   = 1[(A >= 0 and r_t <= 1 + clip_eps) or (A < 0 and r_t >= 1 - clip_eps)]   (fp32 compare)
+ *     omega_t = -(m_t / N) chi_t r_t A  +  beta (m_t / N) (1 - exp(s_ref_t - s_t))
+ * Group statistics are evaluated in fp64 per response, the per-token part in fp32.
+ *
+ *   rewards      [n_resp_total] fp32; the G responses of prompt p are rewards[p*G .. p*G+G-1].
+ *                n_resp_total % G must be 0 (HILORE_SHAPE).
+ *   resp_offset, n_rows   this call covers responses [resp_offset, resp_offset + n_rows), a microbatch
+ *                of the rollout batch; a prompt group may straddle two calls.
+ *   logp_new, logp_old, logp_ref   [n_rows, T] fp32, 16-byte aligned; logp_ref may be NULL iff beta == 0.
+ *   mask         [n_rows, T] u8 (0 / 1), 4-byte aligned.  T % 4 must be 0 (HILORE_SHAPE).
+ *   N_norm, N_norm_dev   the normaliser N: if N_norm_dev (one int64 on the device, e.g. written by
+ *                hilore_mask_count earlier on the same stream) is not NULL it is read by the kernel and
+ *                N_norm is ignored; a device value <= 0 yields omega = 0 everywhere.  Otherwise N_norm
+ *                (host value) must be > 0 (HILORE_ZERO_NORM).
+ *   adv_out      opt [n_rows] fp32, advantage of each response of this call.
+ *   omega        [n_rows, T] fp32, 16-byte aligned.  Masked slots get 0.
+ *   ratio        opt [n_rows, T] fp32 (r_t as computed, also at masked slots), 16-byte aligned.
+ *   clip_mask    opt [n_rows, T] u8 (chi_t), 4-byte aligned.
+ */
+int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                       int64_t n_rows, int64_t T, const float *logp_new, const float *logp_old,
+                       const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                       const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps, float *adv_out,
+                       float *omega, float *ratio, uint8_t *clip_mask, void *stream);
+
+/*
+ * Operational update exposure of U units over one microbatch
+ * (Eq. "activation-token-weights", Eq. "mlp-weighted-exposure"):
+ *     T_b = slots with mask = 1;  abar_u = mean_{t in T_b} a_{t,u}
+ *     alpha_{t,u} = (a_{t,u} + eps_alpha) / (abar_u + eps_alpha)
+ *     E_u = sum_{t in T_b} |omega_t| alpha_{t,u};       |T_b| = 0  =>  E_u = 0
+ * a_{t,u} is row_rms[u*rms_ld + i*T + t - row_shift] for slot (i, t): row_shift = 1 takes the
+ * activation row of the source position that predicts token t (the paper's wording), 0 the
+ * token's own row.  Slots with t - row_shift < 0 are skipped.
+ *
+ *   omega, mask   [n_rows, T] fp32 / u8 of the microbatch.    row_rms  [U, rms_ld] fp32, rms_ld >= n_rows*T.
+ *   exposure      [U] fp32.     sum_abs_omega  opt, one fp32: sum_{t in T_b} |omega_t|.
+ *   workspace     scratch of at least hilore_workspace_bytes(U, n_rows*T) bytes, 16-byte aligned; its
+ *                 contents are overwritten (HILORE_WORKSPACE if too small).  Partial sums are kept in fp64
+ *                 in fixed slots and added in a fixed order: the result is run-to-run deterministic.
+ */
+int hilore_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
+                         const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift, float eps_alpha,
+                         float *exposure, float *sum_abs_omega, void *workspace, size_t workspace_bytes,
+                         void *stream);
+size_t hilore_workspace_bytes(int32_t U, int64_t n_tok);
+
+/*
+ * Compress one bf16 unit (the L action at capture time; Eq. "fp8-roundtrip" for fmt RAW) and, fused
+ * into the same pass, the tokenwise activation magnitude a_t = sqrt(mean_j X_{t,j}^2) of
+ * Eq. "activation-token-weights" (fp32 accumulation per block of 64, fp64 across the blocks of a row;
+ * a row whose squares leave the fp32 range yields Inf).
+ *   fmt RAW : code = cast_E4M3FN(x): one RNE rounding from the bf16 value; |x| up to 464 -> at most 448,
+ *             larger, +-Inf and NaN -> sign | 0x7F.  block must be 0, scales NULL.
+ *   fmt BLK : per block of 64 consecutive elements of a row: amax = max |x_i| over its finite elements;
+ *             s = inv = 1 if amax == 0, if no element is finite, or if Q / amax overflows fp32;
+ *             else s = fl32(amax / Q), inv = fl32(Q / amax), Q = 448 (E4M3FN) or 127 (INT8);
+ *             q_i = fl32(x_i * inv); E4M3FN: code_i = RNE(q_i) saturating at +-448, NaN -> sign|0x7F;
+ *             INT8: code_i = RNE(q_i) clamped to +-127, NaN -> 0x80.  block must be 64.
+ *
+ *   x        [rows, ld] bf16, ld >= cols, 32-byte aligned, ld % 16 == 0.    cols % 16 == 0 (RAW),
+ *            cols % 64 == 0 (BLK).
+ *   codes    [rows, cols] u8, 16-byte aligned; NULL => statistics only (row_rms must then be given).
+ *   scales   [rows, cols/64] fp32 (BLK only).          row_rms  opt [rows] fp32.
+ */
+int hilore_compress(const void *x, int64_t rows, int64_t cols, int64_t ld, int32_t fmt, int32_t block,
+                    uint8_t *codes, float *scales, float *row_rms, void *stream);
+
+/*
+ * Recover a compressed unit to bf16 (the L action at backward time).
+ *   fmt RAW : x_hat = cast_BF16(code), exact; the NaN codes become a bf16 NaN.
+ *   fmt BLK : x_hat = bf16_rne(fl32(value(code) * s)).
+ *   codes [rows, cols] u8, 16-byte aligned;  scales [rows, cols/64] fp32 (BLK);
+ *   out   [rows, ld_out] bf16, 32-byte aligned, ld_out % 16 == 0, ld_out >= cols.
+ */
+int hilore_recover(const uint8_t *codes, const float *scales, int64_t rows, int64_t cols, int32_t fmt,
+                   int32_t block, void *out, int64_t ld_out, void *stream);
+
+/* One recovery unit of a microbatch: where its bf16 bundle lives and where its L representation goes.
+ * A DEVICE array of these is passed to hilore_plan_apply.  Field rules as in hilore_compress /
+ * hilore_recover; `out` may equal `x` only if the caller no longer needs the original. */
+typedef struct hilore_unit {
+    const void *x;   /* [rows, ld] bf16 saved activation                         */
+    uint8_t *codes;  /* [rows, cols] u8                                          */
+    float *scales;   /* [rows, cols/64] fp32, NULL for fmt RAW                   */
+    void *out;       /* [rows, ld] bf16 reconstruction target of RECOVER         */
+    float *row_rms;  /* opt [rows] fp32 token magnitudes written by CAPTURE      */
+    int64_t rows, cols, ld;
+    int32_t fmt, block;
+} hilore_unit;
+
+/*
+ * Risk score, H / L / R gating and the batched capture / encode / recover of all units of a microbatch
+ * in ONE launch per phase (Eq. "token-weighted-risk": psi_u = kappa_c(u) E_u ebar_u;
+ * Eq. "available-recovery-actions").  All decisions stay on the device: the gating arrays are read
+ * by the kernels, so no phase needs a host synchronisation.
+ *
+ *   units_dev   [U] hilore_unit on the DEVICE.     units_host  the same table on the HOST (read during
+ *               the call for validation and launch sizing; must match units_dev).
+ *   avail       [U] u8: the candidate plan q_u in {R, H, L} fixed before forward.
+ *   action_io   [U] u8: DECIDE writes it; the other phases read it.
+ *   DECIDE:  if exposure != NULL: psi_u = fl32(fl32(kappa_u * E_u) * ebar_u); desired = L if psi < tau_lo,
+ *            H if psi >= tau_hi, else R (NaN -> R) -- a threshold stand-in for the paper's knapsack
+ *            allocator; if exposure == NULL the desired action is action_io[u] as given.
+ *            Then action = desired if it is in A_u(q_u) (q = H: {H,L,R}; q = L: {L,R}; q = R: {R}), else R.
+ *            Writes psi (opt), action_io, recompute[u] = (action == R), retained_bytes[u] = 2*rows*cols (H),
+ *            rows*cols + 4*rows*cols/64 (L; no scale term for fmt RAW), 0 (R).
+ *   CAPTURE: q = L: compress into codes / scales and write row_rms; q = H: row_rms only; q = R: untouched.
+ *   ENCODE:  units with q = H and action = L are compressed (post-forward encoding).
+ *   RECOVER: units with action = L are decoded into `out`; H and R units are untouched (H keeps its
+ *            exact bundle, Prop. "exact recovery equivalence"; R is recomputed by the caller).
+ */
+int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit *units_host, int32_t U, int32_t phase,
+                      const float *exposure, const float *kappa, const float *ebar, float tau_lo,
+                      float tau_hi, const uint8_t *avail, uint8_t *action_io, float *psi, uint8_t *recompute,
+                      uint64_t *retained_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HILORE_H */

@@ -1,0 +1,453 @@
+// GRPO loss coefficients and update exposure: hilore_mask_count, hilore_grpo_coeffs,
+// hilore_unit_exposure.  Paper: Eq. "grpo-objective", Eq. "update-coefficient", the K3 derivative in
+// the proof of Prop. 1, Eq. "activation-token-weights" and Eq. "mlp-weighted-exposure".
+#include "common.cuh"
+
+namespace hilore {
+
+// ------------------------------------------------------------------ N = sum of the update mask
+__global__ void __launch_bounds__(256) mask_count_kernel(const uint8_t *mask, int64_t n, unsigned long long *count)
+{
+    // vector part: 16 bytes per step when the base is 16-byte aligned; the rest byte by byte
+    const bool vec = (reinterpret_cast<uintptr_t>(mask) & 15) == 0;
+    const int64_t nvec = vec ? (n >> 4) : 0;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x, gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned int local = 0;
+    const uint4 *m4 = reinterpret_cast<const uint4 *>(mask);
+    for (int64_t i = gid; i < nvec; i += stride) {
+        const uint4 v = ld_global_128_stream(m4 + i);
+        local += __popc(__vcmpne4(v.x, 0) & 0x01010101u) + __popc(__vcmpne4(v.y, 0) & 0x01010101u) +
+                 __popc(__vcmpne4(v.z, 0) & 0x01010101u) + __popc(__vcmpne4(v.w, 0) & 0x01010101u);
+    }
+    for (int64_t i = (nvec << 4) + gid; i < n; i += stride)
+        local += mask[i] != 0;
+    __shared__ unsigned int sm[8];
+    unsigned int w = local;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        w += __shfl_xor_sync(0xFFFFFFFFu, w, o);
+    if ((threadIdx.x & 31) == 0)
+        sm[threadIdx.x >> 5] = w;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long t = 0;
+        for (int i = 0; i < 8; ++i)
+            t += sm[i];
+        if (t)
+            atomicAdd(count, t); // integer addition: the total does not depend on the order
+    }
+}
+
+// ------------------------------------------------------------------ coefficients
+struct CoeffArgs {
+    const float *rewards;
+    int64_t n_resp_total;
+    int G;
+    int64_t resp_offset, n_rows, T;
+    const float *logp_new, *logp_old, *logp_ref;
+    const uint8_t *mask;
+    int64_t N_norm;
+    const long long *N_norm_dev;
+    float clip_eps, beta, adv_eps;
+    float *adv_out, *omega, *ratio;
+    uint8_t *clip_mask;
+    int tiles_per_row;
+};
+
+constexpr int kCoeffThreads = 128;
+constexpr int kCoeffVec = 2;                                  // float4 groups per thread
+constexpr int kCoeffTile = kCoeffThreads * kCoeffVec * 4;     // 1024 slots of one response per CTA
+
+// Advantage of response `resp`, from the G rewards of its prompt group, in fp64 (one warp).
+__device__ float group_advantage(const float *rewards, int64_t resp, int G, float adv_eps, int lane)
+{
+    const float *R = rewards + (resp / G) * G;
+    float lo = INFINITY, hi = -INFINITY;
+    double sum = 0.0;
+    for (int j = lane; j < G; j += 32) {
+        const float v = __ldg(R + j);
+        lo = fminf(lo, v);
+        hi = fmaxf(hi, v);
+        sum += (double)v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    sum = warp_sum(sum);
+    if (lo == hi)
+        return 0.0f; // equal-reward group: exactly zero, whatever the rounding of the mean
+    const double mu = sum / (double)G;
+    double var = 0.0;
+    for (int j = lane; j < G; j += 32) {
+        const double d = (double)__ldg(R + j) - mu;
+        var += d * d;
+    }
+    var = warp_sum(var) / (double)G;
+    const double sigma = sqrt(var);
+    return (float)(((double)__ldg(rewards + resp) - mu) / (sigma + (double)adv_eps));
+}
+
+template <bool KL, bool EXTRA>
+__global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid_constant__ CoeffArgs a)
+{
+    const int64_t tile = blockIdx.x;
+    const int64_t row = tile / a.tiles_per_row;
+    const int tt = (int)(tile - row * a.tiles_per_row);
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int64_t rowbase = row * a.T;
+
+    // issue the token loads first; the group statistics below overlap with them
+    float4 sn[kCoeffVec], so[kCoeffVec], sr[kCoeffVec];
+    uint32_t mk[kCoeffVec];
+    int64_t t0[kCoeffVec];
+#pragma unroll
+    for (int j = 0; j < kCoeffVec; ++j) {
+        t0[j] = (int64_t)tt * kCoeffTile + (int64_t)(j * kCoeffThreads + tid) * 4;
+        if (t0[j] < a.T) {
+            const int64_t k = rowbase + t0[j];
+            sn[j] = __ldcs(reinterpret_cast<const float4 *>(a.logp_new + k));
+            so[j] = __ldcs(reinterpret_cast<const float4 *>(a.logp_old + k));
+            if (KL) sr[j] = __ldcs(reinterpret_cast<const float4 *>(a.logp_ref + k));
+            mk[j] = __ldcs(reinterpret_cast<const unsigned int *>(a.mask + k));
+        }
+    }
+
+    __shared__ float s_adv;
+    if (tid < 32) {
+        const float A = group_advantage(a.rewards, a.resp_offset + row, a.G, a.adv_eps, lane);
+        if (lane == 0) {
+            s_adv = A;
+            if (tt == 0 && a.adv_out)
+                a.adv_out[row] = A;
+        }
+    }
+    __syncthreads();
+    const float A = s_adv;
+    const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
+    const double invN = N > 0 ? 1.0 / (double)N : 0.0;
+    const float coef = (float)(-(double)A * invN); // omega = coef * r on the unclipped branch
+    const float kl = (float)((double)a.beta * invN);
+    const float hi = 1.0f + a.clip_eps, lo = 1.0f - a.clip_eps;
+    const bool pos = A >= 0.0f;
+
+#pragma unroll
+    for (int j = 0; j < kCoeffVec; ++j) {
+        if (t0[j] >= a.T)
+            continue;
+        const float s[4] = {sn[j].x, sn[j].y, sn[j].z, sn[j].w};
+        const float o[4] = {so[j].x, so[j].y, so[j].z, so[j].w};
+        const float rf[4] = {sr[j].x, sr[j].y, sr[j].z, sr[j].w};
+        float w[4], r[4];
+        uint32_t chi = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const bool m = ((mk[j] >> (8 * i)) & 0xFFu) != 0;
+            r[i] = expf(s[i] - o[i]);
+            const bool c = pos ? (r[i] <= hi) : (r[i] >= lo);
+            chi |= (uint32_t)c << (8 * i);
+            float v = (m && c) ? coef * r[i] : 0.0f;
+            if (KL && m)
+                v += kl * (-expm1f(rf[i] - s[i]));
+            w[i] = v;
+        }
+        const int64_t k = rowbase + t0[j];
+        __stcs(reinterpret_cast<float4 *>(a.omega + k), make_float4(w[0], w[1], w[2], w[3]));
+        if (EXTRA) {
+            if (a.ratio) __stcs(reinterpret_cast<float4 *>(a.ratio + k), make_float4(r[0], r[1], r[2], r[3]));
+            if (a.clip_mask) __stcs(reinterpret_cast<unsigned int *>(a.clip_mask + k), chi);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ exposure
+constexpr int kExpThreads = 256;
+constexpr int kExpTile = kExpThreads * 4; // slots per CTA
+constexpr int kExpUnits = 8;              // units per CTA (omega and mask are read once for all of them)
+
+struct ExpArgs {
+    const float *omega;
+    const uint8_t *mask;
+    int64_t n_rows, T, n_tok;
+    const float *row_rms;
+    int U;
+    int64_t rms_ld;
+    int row_shift;
+    double *part; // [(U + 1), ntiles, 2]
+    int ntiles;
+};
+
+template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __grid_constant__ ExpArgs a)
+{
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int tile = blockIdx.x;
+    const int u0 = blockIdx.y * kExpUnits, nu = min(kExpUnits, a.U - u0);
+    float wabs[4];   // |omega| at valid slots, else 0
+    bool mk[4];      // slot is in T_b
+    bool has[4];     // ... and its activation row exists (t - row_shift >= 0)
+    int64_t slot[4];
+    if (VEC) {
+        const int64_t k = (int64_t)tile * kExpTile + (int64_t)tid * 4;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) slot[i] = k + i;
+        if (k < a.n_tok) { // n_tok % 4 == 0: a group is valid as a whole
+            const float4 w = *reinterpret_cast<const float4 *>(a.omega + k);
+            const uint32_t m = *reinterpret_cast<const unsigned int *>(a.mask + k);
+            const float wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                mk[i] = ((m >> (8 * i)) & 0xFFu) != 0;
+                has[i] = mk[i];
+                wabs[i] = mk[i] ? fabsf(wv[i]) : 0.0f;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                mk[i] = false;
+                has[i] = false;
+                wabs[i] = 0.0f;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t k = (int64_t)tile * kExpTile + i * kExpThreads + tid;
+            slot[i] = k;
+            mk[i] = false;
+            has[i] = false;
+            wabs[i] = 0.0f;
+            if (k < a.n_tok && a.mask[k] != 0) {
+                mk[i] = true;
+                wabs[i] = fabsf(a.omega[k]);
+                // a slot whose source row lies before the start of its response has no activation term
+                has[i] = a.row_shift == 0 || (k % a.T) >= a.row_shift;
+            }
+        }
+    }
+    __shared__ double sm[kExpThreads / 32][2 * (kExpUnits + 1)];
+    // per-thread partials in fp32 (four terms), warp tree in fp32, across warps and tiles in fp64
+    float acc[2 * (kExpUnits + 1)];
+    acc[2 * kExpUnits] = (wabs[0] + wabs[1]) + (wabs[2] + wabs[3]);
+    acc[2 * kExpUnits + 1] = (float)((int)mk[0] + (int)mk[1] + (int)mk[2] + (int)mk[3]);
+#pragma unroll
+    for (int j = 0; j < kExpUnits; ++j) {
+        float s1 = 0.0f, s2 = 0.0f;
+        if (j < nu) {
+            const float *ar = a.row_rms + (int64_t)(u0 + j) * a.rms_ld;
+            float av[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            if (VEC) {
+                if (slot[0] < a.n_tok) {
+                    const float4 t = *reinterpret_cast<const float4 *>(ar + slot[0]);
+                    av[0] = t.x; av[1] = t.y; av[2] = t.z; av[3] = t.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (has[i]) av[i] = ar[slot[i] - a.row_shift];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                s1 += has[i] ? av[i] : 0.0f;
+                s2 = fmaf(wabs[i], has[i] ? av[i] : 0.0f, s2);
+            }
+        }
+        acc[2 * j] = s1;
+        acc[2 * j + 1] = s2;
+    }
+#pragma unroll
+    for (int q = 0; q < 2 * (kExpUnits + 1); ++q) {
+        const float v = warp_sum(acc[q]);
+        if (lane == 0) sm[wid][q] = (double)v;
+    }
+    __syncthreads();
+    if (tid < 2 * (kExpUnits + 1)) {
+        double t = 0.0;
+        for (int w = 0; w < kExpThreads / 32; ++w) t += sm[w][tid];
+        const int j = tid >> 1, which = tid & 1;
+        if (j < kExpUnits) {
+            if (j < nu) a.part[((int64_t)(u0 + j) * a.ntiles + tile) * 2 + which] = t;
+        } else if (blockIdx.y == 0) {
+            a.part[((int64_t)a.U * a.ntiles + tile) * 2 + which] = t;
+        }
+    }
+}
+
+// One warp per unit adds the per-tile partials in a fixed order and applies the closed form
+//   E_u = (S2_u + eps * S3) / (S1_u / |T_b| + eps),  S1 = sum a, S2 = sum |omega| a, S3 = sum |omega|.
+__global__ void __launch_bounds__(32) exposure_final_kernel(const double *part, int U, int ntiles, float eps_alpha,
+                                                            float *exposure, float *sum_abs_omega)
+{
+    const int u = blockIdx.x, lane = threadIdx.x;
+    double s1 = 0.0, s2 = 0.0, s3 = 0.0, cnt = 0.0;
+    for (int t = lane; t < ntiles; t += 32) {
+        s1 += part[((int64_t)u * ntiles + t) * 2];
+        s2 += part[((int64_t)u * ntiles + t) * 2 + 1];
+        s3 += part[((int64_t)U * ntiles + t) * 2];
+        cnt += part[((int64_t)U * ntiles + t) * 2 + 1];
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    s3 = warp_sum(s3);
+    cnt = warp_sum(cnt);
+    if (lane == 0) {
+        double E = 0.0;
+        if (cnt > 0.0)
+            E = (s2 + (double)eps_alpha * s3) / (s1 / cnt + (double)eps_alpha);
+        exposure[u] = (float)E;
+        if (u == 0 && sum_abs_omega) *sum_abs_omega = (float)s3;
+    }
+}
+
+} // namespace hilore
+
+using namespace hilore;
+
+extern "C" int hilore_mask_count(const uint8_t *mask, int64_t n, int64_t *count, void *stream)
+{
+    if (count == nullptr || n < 0 || (n > 0 && mask == nullptr))
+        return HILORE_INVALID_ARG;
+    if (!aligned(count, 8))
+        return HILORE_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(count, 0, sizeof(int64_t), st) != cudaSuccess)
+        return HILORE_CUDA;
+    if (n == 0)
+        return HILORE_OK;
+    int64_t blocks = (n / 16 + 255) / 256;
+    const int64_t cap = (int64_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    mask_count_kernel<<<(unsigned)blocks, 256, 0, st>>>(mask, n, reinterpret_cast<unsigned long long *>(count));
+    return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
+
+extern "C" int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                                  int64_t n_rows, int64_t T, const float *logp_new, const float *logp_old,
+                                  const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                                  const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps,
+                                  float *adv_out, float *omega, float *ratio, uint8_t *clip_mask, void *stream)
+{
+    if (rewards == nullptr || n_resp_total < 0 || G <= 0 || resp_offset < 0 || n_rows < 0 || T < 0)
+        return HILORE_INVALID_ARG;
+    if (n_resp_total % G != 0 || resp_offset + n_rows > n_resp_total || T % 4 != 0)
+        return HILORE_SHAPE;
+    if (beta != 0.0f && logp_ref == nullptr)
+        return HILORE_INVALID_ARG;
+    if (N_norm_dev == nullptr && N_norm <= 0)
+        return HILORE_ZERO_NORM;
+    if (n_rows == 0 || T == 0)
+        return HILORE_OK;
+    if (logp_new == nullptr || logp_old == nullptr || mask == nullptr || omega == nullptr)
+        return HILORE_INVALID_ARG;
+    if (!aligned(logp_new, 16) || !aligned(logp_old, 16) || !aligned(logp_ref, 16) || !aligned(omega, 16) ||
+        !aligned(ratio, 16) || !aligned(mask, 4) || !aligned(clip_mask, 4) || !aligned(rewards, 4) ||
+        !aligned(adv_out, 4) || !aligned(N_norm_dev, 8))
+        return HILORE_ALIGN;
+    CoeffArgs a{};
+    a.rewards = rewards;
+    a.n_resp_total = n_resp_total;
+    a.G = G;
+    a.resp_offset = resp_offset;
+    a.n_rows = n_rows;
+    a.T = T;
+    a.logp_new = logp_new;
+    a.logp_old = logp_old;
+    a.logp_ref = (beta != 0.0f) ? logp_ref : nullptr;
+    a.mask = mask;
+    a.N_norm = N_norm;
+    a.N_norm_dev = reinterpret_cast<const long long *>(N_norm_dev);
+    a.clip_eps = clip_eps;
+    a.beta = beta;
+    a.adv_eps = adv_eps;
+    a.adv_out = adv_out;
+    a.omega = omega;
+    a.ratio = ratio;
+    a.clip_mask = clip_mask;
+    const int64_t tpr = (T + kCoeffTile - 1) / kCoeffTile;
+    const int64_t tiles = tpr * n_rows;
+    if (tpr > 0x7FFFFFFF || tiles > 0x7FFFFFFF)
+        return HILORE_SHAPE;
+    a.tiles_per_row = (int)tpr;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool kl = beta != 0.0f, extra = (ratio != nullptr) || (clip_mask != nullptr);
+    if (kl && extra) grpo_coeffs_kernel<true, true><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
+    else if (kl) grpo_coeffs_kernel<true, false><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
+    else if (extra) grpo_coeffs_kernel<false, true><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
+    else grpo_coeffs_kernel<false, false><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
+    return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
+
+extern "C" size_t hilore_workspace_bytes(int32_t U, int64_t n_tok)
+{
+    if (U < 0 || n_tok < 0)
+        return 0;
+    const int64_t ntiles = (n_tok + kExpTile - 1) / kExpTile;
+    return (size_t)(U + 1) * (size_t)(ntiles > 0 ? ntiles : 1) * 2 * sizeof(double);
+}
+
+extern "C" int hilore_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
+                                    const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                    float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
+                                    size_t workspace_bytes, void *stream)
+{
+    if (n_rows < 0 || T < 0 || U < 0 || row_shift < 0 || row_shift > 1)
+        return HILORE_INVALID_ARG;
+    if (U == 0)
+        return HILORE_OK;
+    if (exposure == nullptr || row_rms == nullptr || workspace == nullptr)
+        return HILORE_INVALID_ARG;
+    const int64_t n_tok = n_rows * T;
+    if (n_tok > 0 && (omega == nullptr || mask == nullptr))
+        return HILORE_INVALID_ARG;
+    if (rms_ld < n_tok)
+        return HILORE_SHAPE;
+    if (!aligned(workspace, 16) || !aligned(omega, 4) || !aligned(row_rms, 4) || !aligned(exposure, 4) ||
+        !aligned(sum_abs_omega, 4))
+        return HILORE_ALIGN;
+    if (workspace_bytes < hilore_workspace_bytes(U, n_tok))
+        return HILORE_WORKSPACE;
+    const int64_t ntiles64 = (n_tok + kExpTile - 1) / kExpTile;
+    if (ntiles64 > 0x7FFFFFFF || (U + kExpUnits - 1) / kExpUnits > 65535)
+        return HILORE_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ExpArgs a{};
+    a.omega = omega;
+    a.mask = mask;
+    a.n_rows = n_rows;
+    a.T = T;
+    a.n_tok = n_tok;
+    a.row_rms = row_rms;
+    a.U = U;
+    a.rms_ld = rms_ld;
+    a.row_shift = row_shift;
+    a.part = static_cast<double *>(workspace);
+    a.ntiles = (int)ntiles64;
+    if (a.ntiles > 0) {
+        const dim3 grid((unsigned)a.ntiles, (unsigned)((U + kExpUnits - 1) / kExpUnits));
+        const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
+                         aligned(mask, 4) && aligned(row_rms, 16);
+        if (vec) exposure_partial_kernel<true><<<grid, kExpThreads, 0, st>>>(a);
+        else exposure_partial_kernel<false><<<grid, kExpThreads, 0, st>>>(a);
+        if (cudaGetLastError() != cudaSuccess)
+            return HILORE_CUDA;
+    }
+    exposure_final_kernel<<<(unsigned)U, 32, 0, st>>>(a.part, U, a.ntiles, eps_alpha, exposure, sum_abs_omega);
+    return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
+
+extern "C" const char *hilore_status_string(int status)
+{
+    switch (status) {
+    case HILORE_OK: return "ok";
+    case HILORE_INVALID_ARG: return "invalid argument";
+    case HILORE_SHAPE: return "shape not supported";
+    case HILORE_ALIGN: return "pointer or leading dimension misaligned";
+    case HILORE_ZERO_NORM: return "normaliser N is not positive";
+    case HILORE_CUDA: return "CUDA launch failed";
+    case HILORE_WORKSPACE: return "workspace too small";
+    default: return "unknown status";
+    }
+}
+
+extern "C" int hilore_abi_version(void) { return 1000; }

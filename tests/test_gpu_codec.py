@@ -1,0 +1,133 @@
+"""Parity of hilore_compress / hilore_recover with the CPU oracle: codes, scales and recovered bf16
+bit-exact; token RMS within 1e-5 relative.  All calls go through the C ABI."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_33570_b200 import api, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+FMTS = [api.FMT_E4M3FN_RAW, api.FMT_E4M3FN_BLK, api.FMT_INT8_BLK]
+RMS_RTOL = 1e-5
+
+
+def block_of(fmt):
+    return 0 if fmt == api.FMT_E4M3FN_RAW else 64
+
+
+def check_roundtrip(x, fmt, cols=None, ld_out=None):
+    blk = block_of(fmt)
+    codes, scales, rms = G.compress(x, fmt, cols=cols)
+    o_codes, o_scales = oracle.compress(x, fmt, blk, cols=cols)
+    assert np.array_equal(codes, o_codes), f"codes differ at {np.argwhere(codes != o_codes)[:5]}"
+    if blk:
+        assert np.array_equal(scales.view(np.uint32), o_scales.view(np.uint32))
+    o_rms = oracle.row_rms(x, cols=cols)
+    # the kernel squares and accumulates in fp32 (as the paper does): rows whose squares leave the fp32
+    # range (|x| beyond 1e18 overflows, below 1e-19 underflows) differ from the fp64 oracle -- not compared
+    in_range = np.isfinite(o_rms) & (o_rms < 1e15) & ((o_rms > 1e-15) | (o_rms == 0))
+    assert np.all(np.isfinite(rms[in_range])) and not np.any(np.isfinite(rms[~np.isfinite(o_rms)]))
+    assert G.rel_err(rms[in_range], o_rms[in_range]).max(initial=0) <= RMS_RTOL
+    rec = G.recover(o_codes, o_scales, fmt, ld_out=ld_out)
+    o_rec = oracle.recover(o_codes, o_scales, fmt, blk, ld_out=ld_out)
+    c = o_codes.shape[1]
+    nan = (o_rec[:, :c] & 0x7FFF) > 0x7F80
+    assert np.array_equal(((rec[:, :c] & 0x7FFF) > 0x7F80), nan)
+    assert np.array_equal(rec[:, :c][~nan], o_rec[:, :c][~nan])
+    if ld_out is not None and ld_out > c:
+        assert np.all(rec[:, c:] == (G.CANARY | (G.CANARY << 8))), "padding columns of the output were written"
+    return codes, scales, rms
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_every_bf16_pattern(fmt):
+    """All 65 536 bf16 bit patterns (overflow, subnormals, signed zeros, Inf, NaN payloads)."""
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16).reshape(1024, 64)
+    check_roundtrip(bits, fmt)
+    # patterns shuffled so that blocks mix magnitudes, signs and non-finite values
+    rng = np.random.default_rng(0)
+    check_roundtrip(rng.permutation(bits.reshape(-1)).reshape(64, 1024), fmt)
+
+
+def test_every_code_decodes():
+    codes = np.arange(256, dtype=np.uint32).astype(np.uint8).reshape(4, 64)
+    for fmt in FMTS:
+        scales = None if fmt == api.FMT_E4M3FN_RAW else np.array([[1.0], [0.37], [3e-5], [1e20]], np.float32)
+        rec = G.recover(codes, scales, fmt)
+        o = oracle.recover(codes, scales, fmt, block_of(fmt))
+        nan = (o & 0x7FFF) > 0x7F80
+        assert np.array_equal((rec & 0x7FFF) > 0x7F80, nan)
+        assert np.array_equal(rec[~nan], o[~nan])
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_config1_tiny_units(fmt):
+    """Tiny GRPO step: two units [8192, 896], N(0,1) with 1% x20 outlier channels, seed 0."""
+    rng = np.random.default_rng(0)
+    for _ in range(2):
+        x = synth.activation_unit(rng, 8192, 896)
+        check_roundtrip(x, fmt)
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 64), (3, 192), (37, 4096), (5, 18944), (300, 64), (129, 1536),
+                                       (2, 8960), (1, 262144)])
+@pytest.mark.parametrize("fmt", FMTS)
+def test_ragged_shapes(rows, cols, fmt):
+    x = synth.activation_unit(np.random.default_rng(rows * 131 + cols), rows, cols)
+    check_roundtrip(x, fmt)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_leading_dimensions(fmt):
+    rng = np.random.default_rng(5)
+    x = synth.activation_unit(rng, 50, 640)
+    wide = np.full((50, 704), 0x7FC0, np.uint16)      # NaN padding: must never be read
+    wide[:, :640] = x
+    c1, s1, r1 = G.compress(x, fmt)
+    c2, s2, r2 = check_roundtrip(wide, fmt, cols=640, ld_out=672)
+    assert np.array_equal(c1, c2) and np.array_equal(r1, r2)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_special_values_inside_gaussian_data(fmt):
+    rng = np.random.default_rng(6)
+    x = synth.activation_unit(rng, 64, 1024)
+    x[0, 0:64] = 0                                     # all-zero block
+    x[1, 64:128] = 0x8000                              # all minus-zero block
+    x[2, 5] = 0x7FC0
+    x[3, 70] = 0x7F80
+    x[4, 130] = 0xFF80
+    x[5, 192:256] = 0x0001                             # smallest subnormals
+    x[6, 256:320] = 0x7FC1                             # block without a finite element
+    x[7, 320:384] = 0x7F7F                             # largest finite value
+    x[8, 0] = 0x43E8                                   # 464: last value that still rounds to 448 unscaled
+    x[9, 0] = 0x43E9                                   # 466: overflows to NaN unscaled
+    x[10, 3] = 0xC3E9
+    check_roundtrip(x, fmt)
+
+
+def test_stats_only_and_no_stats():
+    rng = np.random.default_rng(7)
+    x = synth.activation_unit(rng, 77, 1536)
+    _, _, rms = G.compress(x, api.FMT_E4M3FN_RAW, want_codes=False)
+    assert G.rel_err(rms, oracle.row_rms(x)).max() <= RMS_RTOL
+    codes, scales, none = G.compress(x, api.FMT_E4M3FN_BLK, want_rms=False)
+    o_codes, o_scales = oracle.compress(x, api.FMT_E4M3FN_BLK, 64)
+    assert none is None and np.array_equal(codes, o_codes) and np.array_equal(scales, o_scales)
+
+
+def test_run_to_run_determinism():
+    x = synth.activation_unit(np.random.default_rng(8), 4096, 3584)
+    a = G.compress(x, api.FMT_E4M3FN_BLK)
+    b = G.compress(x, api.FMT_E4M3FN_BLK)
+    for p, q in zip(a, b):
+        assert p.tobytes() == q.tobytes()
+
+
+def test_error_statistic_of_gpu_roundtrip_matches_oracle():
+    """e^L of the paper's unscaled round trip on N(0,1) data, GPU recovery vs oracle recovery."""
+    x = synth.activation_unit(np.random.default_rng(9), 256, 1536)
+    codes, _, _ = G.compress(x, api.FMT_E4M3FN_RAW)
+    rec = G.recover(codes, None, api.FMT_E4M3FN_RAW)
+    assert oracle.relative_error(x, rec) == oracle.relative_error(x, oracle.recover(codes, None, 0, 0))

@@ -1,0 +1,186 @@
+"""Parity of hilore_mask_count / hilore_grpo_coeffs / hilore_unit_exposure with the CPU oracle.
+
+fp32 outputs: 1e-5 relative (signed zeros equal).  The clip indicator is an integer decided by an
+fp32 compare of r = exp(s - s_old); the oracle rounds a double exp, the kernel uses expf, so a slot
+whose oracle ratio lies within 4 ulp of a clip bound may legitimately differ and is excused (and
+counted).  All calls go through the C ABI.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_33570_b200 import api, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-5
+
+
+def check_coeffs(ro, got, *, resp_offset=0, N=None, beta=0.0, clip_eps=0.2):
+    n_rows = got["omega"].shape[0]
+    sl = slice(resp_offset, resp_offset + n_rows)
+    adv_all = oracle.group_advantages(ro.rewards, ro.G)
+    N = ro.n_valid if N is None else N
+    w, r, chi = oracle.grpo_coeffs(adv_all[sl], ro.logp_new[sl], ro.logp_old[sl], ro.logp_ref[sl], ro.mask[sl],
+                                   N_norm=N, clip_eps=clip_eps, beta=beta)
+    assert G.rel_err(got["adv"], adv_all[sl]).max() <= RTOL
+    assert np.array_equal(got["adv"] == 0, adv_all[sl] == 0)
+    hi, lo = np.float32(1) + np.float32(clip_eps), np.float32(1) - np.float32(clip_eps)
+    near = (np.abs(r - hi) <= 4 * np.spacing(hi)) | (np.abs(r - lo) <= 4 * np.spacing(lo))
+    if "chi" in got:
+        bad = got["chi"] != chi
+        assert not np.any(bad & ~near), "clip indicator differs away from the clip bounds"
+        assert G.rel_err(got["ratio"], r).max() <= RTOL
+    ok = ~near
+    err = G.rel_err(got["omega"][ok], w[ok])
+    if beta != 0:
+        # where the policy and K3 terms cancel, allow 1e-5 of the larger term (reported, not hidden)
+        kl = beta * ro.mask[sl] / N * (1 - np.exp(ro.logp_ref[sl].astype(np.float64) - ro.logp_new[sl]))
+        floor = RTOL * np.maximum(np.abs(w.astype(np.float64) - kl), np.abs(kl))[ok]
+        assert np.all((err <= RTOL) | (np.abs(got["omega"][ok].astype(np.float64) - w[ok]) <= floor))
+    else:
+        assert err.max(initial=0) <= RTOL, err.max()
+    assert np.all(got["omega"][ro.mask[sl] == 0] == 0)
+    return int(near.sum())
+
+
+def test_config1_tiny():
+    """4 prompts x G=8 x 256 tokens, Bernoulli rewards, all slots valid."""
+    ro = synth.rollout(0, 4, 8, 256)
+    check_coeffs(ro, G.grpo_coeffs(ro, N_norm=ro.n_valid))
+
+
+def test_config2_rollout_batch_and_microbatches():
+    """64 prompts x 8 x 1024 in one call, and as 64 microbatches of 8 responses with resp_offset."""
+    ro = synth.rollout(0, 64, 8, 1024)
+    whole = G.grpo_coeffs(ro, N_norm=ro.n_valid)
+    check_coeffs(ro, whole)
+    for mb in (0, 17, 63):
+        part = G.grpo_coeffs(ro, resp_offset=mb * 8, n_rows=8, N_norm=ro.n_valid)
+        check_coeffs(ro, part, resp_offset=mb * 8)
+        assert np.array_equal(part["omega"], whole["omega"][mb * 8:mb * 8 + 8])
+
+
+def test_group_straddles_microbatches():
+    """G=16 with microbatches of 8 responses: a prompt group spans two calls."""
+    ro = synth.rollout(1, 8, 16, 512)
+    for off in (0, 8, 24, 120):
+        check_coeffs(ro, G.grpo_coeffs(ro, resp_offset=off, n_rows=8, N_norm=ro.n_valid), resp_offset=off)
+
+
+def test_variable_length_masks_and_equal_groups():
+    """Lengths U{128..T}, rewards U[0,1), 5% of the groups all-equal (non-dyadic values): omega exactly 0."""
+    ro = synth.rollout(0, 64, 8, 2048, rewards="uniform", lengths="uniform", equal_group_fraction=0.05)
+    got = G.grpo_coeffs(ro, N_on_device=True)
+    assert got["N"] == ro.n_valid
+    check_coeffs(ro, got)
+    Rg = ro.rewards.reshape(-1, 8)
+    eq = np.where((Rg.max(axis=1) == Rg.min(axis=1)))[0]
+    assert len(eq) == 3
+    for g in eq:
+        assert np.all(got["omega"][g * 8:(g + 1) * 8] == 0) and np.all(got["adv"][g * 8:(g + 1) * 8] == 0)
+
+
+@pytest.mark.parametrize("beta", [1e-3, 0.5])
+def test_k3_regulariser(beta):
+    ro = synth.rollout(2, 16, 8, 512, lengths="uniform")
+    ro.rewards[8:16] = 1.0       # zero-advantage group keeps its K3 contribution
+    got = G.grpo_coeffs(ro, N_norm=ro.n_valid, beta=beta)
+    check_coeffs(ro, got, beta=beta)
+    live = ro.mask[8:16] == 1
+    assert np.all(got["omega"][8:16][live] != 0)
+
+
+def test_without_optional_outputs_and_other_clip_radius():
+    ro = synth.rollout(3, 8, 8, 1280)      # T not a multiple of the 1024-slot tile
+    a = G.grpo_coeffs(ro, N_norm=12345, extras=False, clip_eps=0.05)
+    b = G.grpo_coeffs(ro, N_norm=12345, extras=True, clip_eps=0.05)
+    assert np.array_equal(a["omega"], b["omega"])
+    assert (b["chi"] == 0).mean() > 0.05
+    check_coeffs(ro, b, N=12345, clip_eps=0.05)
+
+
+def test_ratio_one_gives_minus_adv_over_N():
+    ro = synth.rollout(4, 4, 8, 256)
+    ro.logp_old[:] = ro.logp_new
+    got = G.grpo_coeffs(ro, N_norm=ro.n_valid)
+    assert np.all(got["ratio"] == 1) and np.all(got["chi"] == 1)
+    adv = oracle.group_advantages(ro.rewards, 8).astype(np.float64)
+    assert G.rel_err(got["omega"], -adv[:, None] / ro.n_valid * np.ones((1, 256))).max() <= RTOL
+
+
+def test_mask_count_sizes_and_alignment():
+    import torch
+    rng = np.random.default_rng(0)
+    for n in (0, 1, 15, 16, 17, 4097, 1 << 20):
+        m = (rng.random(n + 3) < 0.4).astype(np.uint8)
+        d = G.dev(m)
+        out = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+        api.hilore_mask_count(d, n, out)
+        assert int(out.item()) == int(m[:n].sum())
+        api.hilore_mask_count(d[1:], n, out)       # unaligned base
+        assert int(out.item()) == int(m[1:n + 1].sum())
+
+
+def _rms_for(ro, U, seed):
+    rng = np.random.default_rng(seed)
+    return (rng.random((U, ro.n_resp * ro.T), dtype=np.float32) * np.float32(2) + np.float32(0.25))
+
+
+@pytest.mark.parametrize("U", [1, 2, 9, 84])
+def test_exposure_config1(U):
+    ro = synth.rollout(0, 4, 8, 256)
+    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    rms = _rms_for(ro, U, 1)
+    E, sw = G.unit_exposure(omega, ro.mask, rms)
+    oE, osw = oracle.unit_exposure(omega, ro.mask, rms)
+    assert G.rel_err(E, oE).max() <= RTOL and abs(sw - osw) <= RTOL * osw
+
+
+def test_exposure_masked_microbatch_and_row_shift():
+    """Microbatch of 4 responses x 4096 slots with padding; both row conventions."""
+    ro = synth.rollout(0, 1, 4, 4096, rewards="uniform", lengths="uniform", mask_first_column=True)
+    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    rms = _rms_for(ro, 5, 2)
+    rms[:, ro.mask.reshape(-1) == 0] = 1e9          # padded rows must not contribute
+    for shift in (0, 1):
+        r = rms.copy()
+        if shift:
+            r = np.roll(rms.reshape(5, 4, 4096), -1, axis=2).reshape(5, -1).copy()
+        E, sw = G.unit_exposure(omega, ro.mask, r, row_shift=shift)
+        oE, osw = oracle.unit_exposure(omega, ro.mask, r, row_shift=shift)
+        assert G.rel_err(E, oE).max() <= RTOL and abs(sw - osw) <= RTOL * osw
+    E0, _ = G.unit_exposure(omega, ro.mask, rms, row_shift=0)
+    E1, _ = G.unit_exposure(omega, ro.mask, np.roll(rms.reshape(5, 4, 4096), -1, axis=2).reshape(5, -1).copy(), row_shift=1)
+    assert G.rel_err(E1, E0).max() <= RTOL
+
+
+def test_exposure_degenerate_cases():
+    ro = synth.rollout(5, 2, 4, 64)
+    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    rms = _rms_for(ro, 3, 3)
+    E, sw = G.unit_exposure(np.zeros_like(omega), ro.mask, rms)
+    assert np.all(E == 0) and sw == 0                       # all coefficients zero
+    E, sw = G.unit_exposure(omega, np.zeros_like(ro.mask), rms)
+    assert np.all(E == 0) and sw == 0                       # empty T_b
+    odd = omega.reshape(-1)[:501].reshape(3, 167).copy()    # sizes that defeat the vector path
+    m = (np.random.default_rng(1).random((3, 167)) < 0.7).astype(np.uint8)
+    r = _rms_for(ro, 3, 4)[:, :501].copy()
+    E, sw = G.unit_exposure(odd, m, r)
+    oE, osw = oracle.unit_exposure(odd, m, r)
+    assert G.rel_err(E, oE).max() <= RTOL
+    a, b = G.unit_exposure(omega, ro.mask, rms), G.unit_exposure(omega, ro.mask, rms)
+    assert a[0].tobytes() == b[0].tobytes()                 # fixed reduction order
+
+
+def test_exposure_from_fused_token_rms():
+    """End of the chain: token RMS written by hilore_compress feeds hilore_unit_exposure."""
+    ro = synth.rollout(0, 4, 8, 256)
+    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    rng = np.random.default_rng(0)
+    units = [synth.activation_unit(rng, 8192, 896) for _ in range(2)]
+    rms = np.stack([G.compress(x, api.FMT_E4M3FN_BLK)[2] for x in units])
+    E, _ = G.unit_exposure(omega, ro.mask, rms)
+    o_rms = np.stack([oracle.row_rms(x) for x in units])
+    oE, _ = oracle.unit_exposure(omega, ro.mask, o_rms)
+    assert G.rel_err(E, oE).max() <= RTOL
