@@ -132,6 +132,32 @@ int hilore_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows
 size_t hilore_workspace_bytes(int32_t U, int64_t n_tok);
 
 /*
+ * hilore_unit_exposure for callers that cannot provide a workspace.  (The paper has no counterpart:
+ * this is a packaging variant of the same reduction, with the same results.)
+ *
+ * Who needs it: code that must not allocate at the point where the exposure refresh runs -- for example
+ * a saved-tensor hook running where the framework's caching allocator may not be re-entered, a process
+ * whose device memory is wholly owned by another pool, or a latency-critical loop in which cudaMalloc
+ * (which may synchronise the device) is ruled out.  The call allocates nothing on host or device: the
+ * fp64 partial sums go to a fixed 1 MiB array inside the library image (hilore_static_scratch_bytes()),
+ * which every GPU context that loads the library holds until it exits.
+ *
+ *   Arguments and results as hilore_unit_exposure, minus the workspace.
+ *   Limit: hilore_workspace_bytes(U, n_rows*T) must not exceed the built-in array, i.e.
+ *   (U + 1) * ceil(n_rows*T / 1024) <= 65536; larger problems return HILORE_WORKSPACE and nothing is
+ *   launched (use hilore_unit_exposure with your own workspace).
+ *   First call on a device: looks up the array's device address (once per device, with that device
+ *   current) -- make this first call outside any stream capture.
+ *   The array is shared by all calls and keeps the previous call's contents; every slot a call reads it
+ *   has written first, so nothing needs clearing.  Two calls that overlap on the GPU (different streams
+ *   without ordering, or several host threads) race on the array: order them.
+ */
+int hilore_unit_exposure_static(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
+                                const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                float eps_alpha, float *exposure, float *sum_abs_omega, void *stream);
+size_t hilore_static_scratch_bytes(void);
+
+/*
  * Compress one bf16 unit (the L action at capture time; Eq. "fp8-roundtrip" for fmt RAW) and, fused
  * into the same pass, the tokenwise activation magnitude a_t = sqrt(mean_j X_{t,j}^2) of
  * Eq. "activation-token-weights" (fp32 accumulation per block of 64, fp64 across the blocks of a row;

@@ -23,7 +23,7 @@ BLOCK = 64
 
 EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "hilore_grpo_coeffs",
            "hilore_unit_exposure", "hilore_workspace_bytes", "hilore_compress", "hilore_recover",
-           "hilore_plan_apply")
+           "hilore_plan_apply", "hilore_unit_exposure_static", "hilore_static_scratch_bytes")
 
 
 class HiloreUnit(C.Structure):
@@ -65,11 +65,14 @@ def lib() -> C.CDLL:
         _lib.hilore_grpo_coeffs.argtypes = [vp, i64, i32, i64, i64, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32,
                                             vp, vp, vp, vp, vp]
         _lib.hilore_unit_exposure.argtypes = [vp, vp, i64, i64, vp, i32, i64, i32, f32, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_unit_exposure_static.argtypes = [vp, vp, i64, i64, vp, i32, i64, i32, f32, vp, vp, vp]
+        _lib.hilore_static_scratch_bytes.restype = C.c_size_t
+        _lib.hilore_static_scratch_bytes.argtypes = []
         _lib.hilore_compress.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
         _lib.hilore_recover.argtypes = [vp, vp, i64, i64, i32, i32, vp, i64, vp]
         _lib.hilore_plan_apply.argtypes = [vp, vp, i32, i32, vp, vp, vp, f32, f32, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
-            if name not in ("hilore_status_string", "hilore_workspace_bytes"):
+            if name not in ("hilore_status_string", "hilore_workspace_bytes", "hilore_static_scratch_bytes"):
                 getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -123,6 +126,19 @@ def hilore_unit_exposure(omega, mask, n_rows, T, row_rms, U, rms_ld, row_shift, 
                                     eps_alpha, _ptr(exposure), _ptr(sum_abs_omega), _ptr(workspace),
                                     workspace_bytes, _stream(stream))
     return _check(st, "hilore_unit_exposure", check)
+
+
+def hilore_static_scratch_bytes():
+    return int(lib().hilore_static_scratch_bytes())
+
+
+def hilore_unit_exposure_static(omega, mask, n_rows, T, row_rms, U, rms_ld, row_shift, eps_alpha, exposure,
+                                sum_abs_omega, stream=None, check=True):
+    """hilore_unit_exposure without a workspace argument: the partial sums use the library's built-in
+    1 MiB scratch array, so the call allocates nothing (see include/hilore.h for the limits)."""
+    st = lib().hilore_unit_exposure_static(_ptr(omega), _ptr(mask), n_rows, T, _ptr(row_rms), U, rms_ld, row_shift,
+                                           eps_alpha, _ptr(exposure), _ptr(sum_abs_omega), _stream(stream))
+    return _check(st, "hilore_unit_exposure_static", check)
 
 
 def hilore_compress(x, rows, cols, ld, fmt, block, codes, scales, row_rms, stream=None, check=True):

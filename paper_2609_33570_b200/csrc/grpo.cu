@@ -451,3 +451,58 @@ extern "C" const char *hilore_status_string(int status)
 }
 
 extern "C" int hilore_abi_version(void) { return 1000; }
+
+// ------------------------------------------------------------------ exposure without caller scratch
+// Some callers cannot hand over a workspace: a saved-tensor hook that runs while the framework's
+// caching allocator must not be entered, a host that has given every byte of device memory to
+// another pool, or a latency-critical loop in which cudaMalloc (which may synchronise the whole
+// device) is forbidden.  For them the partial sums of the exposure reduction live in a fixed array
+// that is part of the library image: every GPU context that loads the library holds these bytes
+// until it exits.
+#include <mutex>
+
+namespace hilore {
+constexpr size_t kStaticScratchBytes = size_t(1) << 20; // 1 MiB: (U + 1) * ceil(n_tok / 1024) <= 65536
+static __device__ __align__(256) unsigned char g_exposure_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mutex;
+static void *g_scratch_addr[kMaxDevices] = {};
+
+// Device address of g_exposure_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, not an address a kernel could use: the address is asked for once per
+// device, with that device current, and cached.
+static int static_scratch_address(void **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return HILORE_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_addr[dev] == nullptr) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_exposure_scratch) != cudaSuccess || p == nullptr)
+            return HILORE_CUDA;
+        g_scratch_addr[dev] = p;
+    }
+    *out = g_scratch_addr[dev];
+    return HILORE_OK;
+}
+} // namespace hilore
+
+extern "C" size_t hilore_static_scratch_bytes(void) { return hilore::kStaticScratchBytes; }
+
+extern "C" int hilore_unit_exposure_static(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
+                                           const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                           float eps_alpha, float *exposure, float *sum_abs_omega, void *stream)
+{
+    if (n_rows < 0 || T < 0 || U < 0)
+        return HILORE_INVALID_ARG;
+    if (hilore_workspace_bytes(U, n_rows * T) > hilore::kStaticScratchBytes)
+        return HILORE_WORKSPACE; // beyond the built-in scratch: use hilore_unit_exposure with a workspace
+    void *scratch = nullptr;
+    const int st = hilore::static_scratch_address(&scratch);
+    if (st != HILORE_OK)
+        return st;
+    return hilore_unit_exposure(omega, mask, n_rows, T, row_rms, U, rms_ld, row_shift, eps_alpha, exposure,
+                                sum_abs_omega, scratch, hilore::kStaticScratchBytes, stream);
+}
