@@ -4,77 +4,67 @@
 // microbatch of units therefore costs one launch per phase and no host synchronisation.
 #include "codec.cuh"
 
+#include <cstdlib>
+#include <cstring>
+
 namespace hilore {
 
-struct CodecWork {
-    const hilore_unit *units; // device table, or nullptr => `single`
-    hilore_unit single;
-    int U;
-    int phase;                // HILORE_PHASE_* for table mode; CodecOp for single mode
-    const uint8_t *avail;     // q_u
-    const uint8_t *action;    // a_u
-};
-
-__device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
+// Compress / token-RMS pass over rows [r0, r1) of one unit, specialised on what the unit asks for.
+template <int FMT>
+__device__ __forceinline__ void compress_unit(const hilore_unit &u, int op, int64_t r0, int64_t r1, float *sm, int pf)
 {
-    if (wk.units == nullptr)
-        return wk.phase;
-    switch (wk.phase) {
-    case HILORE_PHASE_CAPTURE: {
-        const uint8_t q = wk.avail[u];
-        return q == HILORE_ACT_L ? OP_COMPRESS : (q == HILORE_ACT_H ? OP_STATS : OP_NONE);
-    }
-    case HILORE_PHASE_ENCODE:
-        return (wk.avail[u] == HILORE_ACT_H && wk.action[u] == HILORE_ACT_L) ? OP_COMPRESS : OP_NONE;
-    case HILORE_PHASE_RECOVER:
-        return wk.action[u] == HILORE_ACT_L ? OP_RECOVER : OP_NONE;
-    default:
-        return OP_NONE;
+    const uint16_t *x = static_cast<const uint16_t *>(u.x);
+    if (op == OP_STATS)
+        compress_rows<HILORE_FMT_E4M3FN_RAW, false, true>(x, nullptr, nullptr, u.row_rms, u.cols, u.ld, r0, r1, sm, pf);
+    else if (u.row_rms != nullptr)
+        compress_rows<FMT, true, true>(x, u.codes, u.scales, u.row_rms, u.cols, u.ld, r0, r1, sm, pf);
+    else
+        compress_rows<FMT, true, false>(x, u.codes, u.scales, nullptr, u.cols, u.ld, r0, r1, sm, pf);
+}
+
+// FMT >= 0: every unit of the launch has this format (the common case; the hot loop is compiled for it).
+// FMT < 0: formats differ between units; each unit is dispatched on its own format.
+template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_kernel(const __grid_constant__ CodecWork wk)
+{
+    __shared__ float sm_blocksum[kBlockSumSlots];
+    Walker w = walker_init(wk);
+    Job j;
+    while (next_job(wk, w, j)) {
+        if (j.op == OP_RECOVER)
+            continue;
+        const int fmt = FMT >= 0 ? FMT : j.u.fmt;
+        if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch);
+        else compress_unit<HILORE_FMT_INT8_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch);
     }
 }
 
-template <int UNR>
-__global__ void __launch_bounds__(kCodecThreads) codec_kernel(const __grid_constant__ CodecWork wk)
+template <int FMT> __device__ __forceinline__ void recover_unit(const hilore_unit &u, int64_t r0, int64_t r1, uint8_t *sm_out,
+                                                                uint32_t &tile, int prefetch)
 {
-    __shared__ float sm_blocksum[kBlockSumSlots];
-    const int64_t nC = gridDim.x, cta = blockIdx.x;
-    for (int ui = 0; ui < wk.U; ++ui) {
-        const int op = unit_op(wk, ui);
-        if (op == OP_NONE)
+    uint16_t *out = static_cast<uint16_t *>(u.out);
+    if (u.ld == u.cols)
+        recover_rows_bulk<FMT>(u.codes, u.scales, out, u.cols, r0, r1, sm_out, tile, prefetch);
+    else
+        recover_rows<FMT>(u.codes, u.scales, out, u.cols, u.ld, r0, r1, prefetch);
+}
+
+template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_kernel(const __grid_constant__ CodecWork wk)
+{
+    __shared__ __align__(128) uint8_t sm_out[kRecoverStageBytes];
+    uint32_t tile = 0;
+    Walker w = walker_init(wk);
+    Job j;
+    while (next_job(wk, w, j)) {
+        if (j.op != OP_RECOVER)
             continue;
-        hilore_unit u = wk.units ? wk.units[ui] : wk.single;
-        // balanced contiguous row ranges: CTA c owns rows [rows*c/nC, rows*(c+1)/nC)
-        const int64_t r0 = (u.rows * cta) / nC, r1 = (u.rows * (cta + 1)) / nC;
-        if (r0 >= r1)
-            continue;
-        const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
-        if ((op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (op == OP_STATS && !u.x) ||
-            (op == OP_RECOVER && (!u.out || !u.codes || (scaled && !u.scales))))
-            continue; // the unit lacks a buffer this operation needs: leave it untouched
-        if (op == OP_STATS) {
-            if (u.row_rms != nullptr)
-                compress_rows<HILORE_FMT_E4M3FN_RAW, false, UNR>(u, r0, r1, sm_blocksum);
-            continue;
-        }
-        if (op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
-            u.row_rms = nullptr; // token magnitudes were collected at capture time
-        switch (u.fmt) {
-        case HILORE_FMT_E4M3FN_RAW:
-            if (op == OP_COMPRESS) compress_rows<HILORE_FMT_E4M3FN_RAW, true, UNR>(u, r0, r1, sm_blocksum);
-            else recover_rows<HILORE_FMT_E4M3FN_RAW, UNR>(u, r0, r1);
-            break;
-        case HILORE_FMT_E4M3FN_BLK:
-            if (op == OP_COMPRESS) compress_rows<HILORE_FMT_E4M3FN_BLK, true, UNR>(u, r0, r1, sm_blocksum);
-            else recover_rows<HILORE_FMT_E4M3FN_BLK, UNR>(u, r0, r1);
-            break;
-        case HILORE_FMT_INT8_BLK:
-            if (op == OP_COMPRESS) compress_rows<HILORE_FMT_INT8_BLK, true, UNR>(u, r0, r1, sm_blocksum);
-            else recover_rows<HILORE_FMT_INT8_BLK, UNR>(u, r0, r1);
-            break;
-        default:
-            break;
-        }
+        const int fmt = FMT >= 0 ? FMT : j.u.fmt;
+        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        else recover_unit<HILORE_FMT_INT8_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
     }
+    if (threadIdx.x == 0)
+        bulk_wait_all(); // every bulk store of this CTA is complete before it gives up its shared memory
 }
 
 // psi, threshold rule, availability demotion, recompute flags and retained bytes for U units.
@@ -136,19 +126,50 @@ static int check_unit(const hilore_unit &u, bool strict, bool need_x, bool need_
     return HILORE_OK;
 }
 
-static int launch_codec(const CodecWork &wk, int64_t max_rows, cudaStream_t st)
+static int env_int(const char *name, int dflt)
 {
-    if (max_rows <= 0)
-        return HILORE_OK;
+    const char *v = std::getenv(name);
+    return v ? std::atoi(v) : dflt;
+}
+
+template <typename K> static int launch_one(K kernel, CodecWork wk, int64_t total_rows, int prefetch, cudaStream_t st)
+{
+    wk.prefetch = prefetch;
+    wk.split_global = env_int("HILORE_SPLIT_GLOBAL", 0);
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, codec_kernel<2>, kCodecThreads, 0) != cudaSuccess ||
-        per_sm <= 0)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kCodecThreads, 0) != cudaSuccess || per_sm <= 0)
         per_sm = 2;
+    const int cap = env_int("HILORE_PER_SM", 0);
+    if (cap > 0 && cap < per_sm)
+        per_sm = cap;
     int64_t grid = (int64_t)sm_count() * per_sm;
-    if (grid > max_rows)
-        grid = max_rows;
-    codec_kernel<2><<<(unsigned)grid, kCodecThreads, 0, st>>>(wk);
+    if (grid > total_rows)
+        grid = total_rows;
+    kernel<<<(unsigned)grid, kCodecThreads, 0, st>>>(wk);
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
+
+// fmt: the format shared by all units of the launch, or -1 if they differ.
+static int launch_codec(const CodecWork &wk, int64_t total_rows, int fmt, bool recover, cudaStream_t st)
+{
+    if (total_rows <= 0)
+        return HILORE_OK;
+    if (recover) {
+        const int pf = env_int("HILORE_PF_R", 0);
+        switch (fmt) {
+        case HILORE_FMT_E4M3FN_RAW: return launch_one(recover_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, pf, st);
+        case HILORE_FMT_E4M3FN_BLK: return launch_one(recover_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, pf, st);
+        case HILORE_FMT_INT8_BLK: return launch_one(recover_kernel<HILORE_FMT_INT8_BLK>, wk, total_rows, pf, st);
+        default: return launch_one(recover_kernel<-1>, wk, total_rows, pf, st);
+        }
+    }
+    const int pf = env_int("HILORE_PF_C", 2);
+    switch (fmt) {
+    case HILORE_FMT_E4M3FN_RAW: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, pf, st);
+    case HILORE_FMT_E4M3FN_BLK: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, pf, st);
+    case HILORE_FMT_INT8_BLK: return launch_one(compress_kernel<HILORE_FMT_INT8_BLK>, wk, total_rows, pf, st);
+    default: return launch_one(compress_kernel<-1>, wk, total_rows, pf, st);
+    }
 }
 
 } // namespace hilore
@@ -180,7 +201,7 @@ extern "C" int hilore_compress(const void *x, int64_t rows, int64_t cols, int64_
     wk.single = u;
     wk.U = 1;
     wk.phase = codes ? OP_COMPRESS : OP_STATS;
-    return launch_codec(wk, rows, static_cast<cudaStream_t>(stream));
+    return launch_codec(wk, rows, fmt, false, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int hilore_recover(const uint8_t *codes, const float *scales, int64_t rows, int64_t cols, int32_t fmt,
@@ -202,7 +223,7 @@ extern "C" int hilore_recover(const uint8_t *codes, const float *scales, int64_t
     wk.single = u;
     wk.U = 1;
     wk.phase = OP_RECOVER;
-    return launch_codec(wk, rows, static_cast<cudaStream_t>(stream));
+    return launch_codec(wk, rows, fmt, true, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit *units_host, int32_t U, int32_t phase,
@@ -217,13 +238,15 @@ extern "C" int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit
     if (units_dev == nullptr || units_host == nullptr || avail == nullptr || action_io == nullptr)
         return HILORE_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int64_t max_rows = 0;
+    int64_t total_rows = 0;
+    int common_fmt = units_host[0].fmt;
     for (int u = 0; u < U; ++u) {
         const int s = check_unit(units_host[u], false, false, false, false);
         if (s != HILORE_OK)
             return s;
-        if (units_host[u].rows > max_rows)
-            max_rows = units_host[u].rows;
+        total_rows += units_host[u].rows;
+        if (units_host[u].fmt != common_fmt)
+            common_fmt = -1;
     }
     if (phase == HILORE_PHASE_DECIDE) {
         if (exposure != nullptr && (kappa == nullptr || ebar == nullptr))
@@ -238,5 +261,5 @@ extern "C" int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit
     wk.phase = phase;
     wk.avail = avail;
     wk.action = action_io;
-    return launch_codec(wk, max_rows, st);
+    return launch_codec(wk, total_rows, common_fmt, phase == HILORE_PHASE_RECOVER, st);
 }

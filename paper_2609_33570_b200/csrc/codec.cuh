@@ -2,11 +2,14 @@
 // and back.  Paper: Eq. "fp8-roundtrip" (unscaled cast) and Eq. "activation-token-weights" (a_t).
 //
 // Work split.  A CTA owns a contiguous range of rows of a unit.  A thread owns 16 consecutive
-// elements ("chunk": one 256-bit load, one 128-bit store of codes); four neighbouring lanes own one
-// 64-element block, so the block absmax and the block sum of squares are two xor-shuffles.  Rows
-// are swept in batches small enough that the per-block sums of squares of a batch fit in shared
-// memory; at the end of a batch each warp adds the blocks of whole rows in a fixed order, so the
-// token RMS is deterministic (no floating-point atomics anywhere).
+// elements ("chunk": one 256-bit load, one 128-bit store of codes) and handles chunks in pairs; four
+// neighbouring lanes own one 64-element block, so the block absmax and the block sum of squares are
+// xor-shuffles inside a quad.  Rows are swept in batches small enough that the per-block sums of
+// squares of a batch fit in shared memory; at the end of a batch each warp adds the blocks of whole
+// rows in a fixed order, so the token RMS is deterministic (no floating-point atomics anywhere).
+// The instruction budget matters: at 6.5 TB/s the SM has about 8 issue slots per element, so the hot
+// loop uses packed bf16x2 maxima, packed f32x2 multiplies / FMAs, one IEEE division per thread and
+// pair of blocks, and pointer increments instead of index arithmetic.
 #pragma once
 
 #include "common.cuh"
@@ -15,8 +18,131 @@ namespace hilore {
 
 enum CodecOp { OP_NONE = 0, OP_COMPRESS = 1, OP_STATS = 2, OP_RECOVER = 3 };
 
+struct CodecWork {
+    const hilore_unit *units; // device table, or nullptr => `single`
+    hilore_unit single;
+    int U;
+    int phase;                // HILORE_PHASE_* for table mode; CodecOp for single mode
+    const uint8_t *avail;     // q_u
+    const uint8_t *action;    // a_u
+    int prefetch;             // iterations of L2 prefetch run-ahead (0 = none)
+    int split_global;         // 1: one slice of the whole launch per CTA; 0: a slice of every unit per CTA
+};
+
+__device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
+{
+    if (wk.units == nullptr)
+        return wk.phase;
+    switch (wk.phase) {
+    case HILORE_PHASE_CAPTURE: {
+        const uint8_t q = wk.avail[u];
+        return q == HILORE_ACT_L ? OP_COMPRESS : (q == HILORE_ACT_H ? OP_STATS : OP_NONE);
+    }
+    case HILORE_PHASE_ENCODE:
+        return (wk.avail[u] == HILORE_ACT_H && wk.action[u] == HILORE_ACT_L) ? OP_COMPRESS : OP_NONE;
+    case HILORE_PHASE_RECOVER:
+        return wk.action[u] == HILORE_ACT_L ? OP_RECOVER : OP_NONE;
+    default:
+        return OP_NONE;
+    }
+}
+
+
+// ---- work split ----
+// The elements of all units a launch is gated into form one stream; CTA c takes the slice
+// [W*c/nC, W*(c+1)/nC) of it, rounded to whole rows.  A CTA therefore streams a few large contiguous
+// pieces (about 1/nC of the launch's bytes) instead of a sliver of every unit.
+struct Job {
+    hilore_unit u;
+    int op;
+    int64_t r0, r1; // this CTA's rows of the unit
+};
+
+__device__ __forceinline__ bool unit_active(const CodecWork &wk, int ui, int &op, hilore_unit &u)
+{
+    op = unit_op(wk, ui);
+    if (op == OP_NONE)
+        return false;
+    u = wk.units ? wk.units[ui] : wk.single;
+    const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
+    if ((op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (op == OP_STATS && (!u.x || !u.row_rms)) ||
+        (op == OP_RECOVER && (!u.out || !u.codes || (scaled && !u.scales))))
+        return false; // the unit lacks a buffer this operation needs: leave it untouched
+    if (op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
+        u.row_rms = nullptr; // token magnitudes were collected at capture time
+    return u.rows > 0;
+}
+
+struct Walker {
+    int64_t lo, hi; // this CTA's slice of the stream of all active elements
+    int64_t off;    // stream offset of the next unit
+    int ui;
+};
+
+__device__ __forceinline__ Walker walker_init(const CodecWork &wk)
+{
+    int64_t W = 0;
+    for (int ui = 0; ui < wk.U; ++ui) {
+        int op;
+        hilore_unit u;
+        if (unit_active(wk, ui, op, u))
+            W += u.rows * u.cols;
+    }
+    Walker w;
+    w.lo = (W / gridDim.x) * blockIdx.x + ((W % gridDim.x) * blockIdx.x) / gridDim.x;
+    w.hi = (W / gridDim.x) * (blockIdx.x + 1) + ((W % gridDim.x) * (blockIdx.x + 1)) / gridDim.x;
+    w.off = 0;
+    w.ui = 0;
+    return w;
+}
+
+// First row of a unit (at stream offset `off`) that belongs to slices starting at stream position x or later:
+// a row goes to the slice that holds its first element.
+__device__ __forceinline__ int64_t row_boundary(int64_t x, int64_t off, int64_t rows, int64_t cols)
+{
+    if (x <= off)
+        return 0;
+    return min((x - off + cols - 1) / cols, rows);
+}
+
+__device__ __forceinline__ bool next_job(const CodecWork &wk, Walker &w, Job &j)
+{
+    for (; w.ui < wk.U; ++w.ui) {
+        if (!unit_active(wk, w.ui, j.op, j.u))
+            continue;
+        if (!wk.split_global) {
+            j.r0 = (j.u.rows * (int64_t)blockIdx.x) / gridDim.x;
+            j.r1 = (j.u.rows * (int64_t)(blockIdx.x + 1)) / gridDim.x;
+            if (j.r0 >= j.r1)
+                continue;
+            ++w.ui;
+            return true;
+        }
+        const int64_t off = w.off;
+        w.off += j.u.rows * j.u.cols;
+        if (off >= w.hi) { // nothing further can intersect this CTA's slice
+            w.ui = wk.U;
+            return false;
+        }
+        j.r0 = row_boundary(w.lo, off, j.u.rows, j.u.cols);
+        j.r1 = row_boundary(w.hi, off, j.u.rows, j.u.cols);
+        if (j.r0 >= j.r1)
+            continue;
+        ++w.ui;
+        return true;
+    }
+    return false;
+}
+
 template <int FMT> struct QMax {
     static constexpr float value = (FMT == HILORE_FMT_INT8_BLK) ? 127.0f : 448.0f;
+};
+
+// Largest |bf16| pattern whose reciprocal scale Q / amax no longer fits fp32 (it rounds to Inf):
+// 448 / (1.75 * 2^-120) = 2^128 and 127 / (1.984375 * 2^-122) = 2^128.  At or below it (zero included)
+// the block takes s = inv = 1.
+template <int FMT> struct UnitScaleBelow {
+    static constexpr uint32_t value = (FMT == HILORE_FMT_INT8_BLK) ? 0x02FEu : 0x03E0u;
 };
 
 __device__ __forceinline__ uint32_t int8_code(float q)
@@ -26,30 +152,36 @@ __device__ __forceinline__ uint32_t int8_code(float q)
     return (uint32_t)v & 0xFFu;
 }
 
-// Sixteen elements, every one finite (BLK) / none above 464 in magnitude (RAW).
-template <int FMT> __device__ __forceinline__ uint4 encode16_fast(const uint32_t (&w)[8], float inv)
+// max.NaN.xorsign.abs.bf16x2: per half, magnitude = max(|a|, |b|) (NaN if either is NaN), sign = junk
+__device__ __forceinline__ uint32_t maxabs_bf16x2(uint32_t a, uint32_t b)
 {
-    uint32_t c[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float e0 = bf16_lo(w[2 * i]), e1 = bf16_hi(w[2 * i]);
-        float e2 = bf16_lo(w[2 * i + 1]), e3 = bf16_hi(w[2 * i + 1]);
-        if (FMT != HILORE_FMT_E4M3FN_RAW) {
-            e0 = __fmul_rn(e0, inv);
-            e1 = __fmul_rn(e1, inv);
-            e2 = __fmul_rn(e2, inv);
-            e3 = __fmul_rn(e3, inv);
-        }
-        if (FMT == HILORE_FMT_INT8_BLK)
-            c[i] = int8_code(e0) | (int8_code(e1) << 8) | (int8_code(e2) << 16) | (int8_code(e3) << 24);
-        else
-            c[i] = cvt_e4m3x2(e1, e0) | (cvt_e4m3x2(e3, e2) << 16);
-    }
-    return make_uint4(c[0], c[1], c[2], c[3]);
+    uint32_t d;
+    asm("max.NaN.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+__device__ __forceinline__ uint32_t maxnan_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// |bf16| bit pattern of the largest magnitude among sixteen elements; 0x7FFF if any of them is NaN,
+// 0x7F80 if any is Inf (and none NaN): one compare against 0x7F80 finds every block that needs care.
+__device__ __forceinline__ uint32_t absmax16(const uint32_t (&w)[8])
+{
+    uint32_t a = maxabs_bf16x2(w[0], w[1]), b = maxabs_bf16x2(w[2], w[3]);
+    uint32_t c = maxabs_bf16x2(w[4], w[5]), d = maxabs_bf16x2(w[6], w[7]);
+    a = maxabs_bf16x2(a, b);
+    c = maxabs_bf16x2(c, d);
+    a = maxabs_bf16x2(a, c);
+    a = maxabs_bf16x2(a, a >> 16);
+    return a & 0x7FFFu;
 }
 
 // One element with the full rule set (overflow, Inf, NaN).  Rare path.
-template <int FMT> __device__ __noinline__ uint32_t encode1_careful(uint32_t bits, float inv)
+template <int FMT> __device__ __forceinline__ uint32_t encode1_careful(uint32_t bits, float inv)
 {
     const uint32_t a = bits & 0x7FFFu, sign = (bits >> 8) & 0x80u;
     const float x = __uint_as_float(bits << 16);
@@ -72,8 +204,10 @@ template <int FMT> __device__ __noinline__ uint32_t encode1_careful(uint32_t bit
     return int8_code(__fmul_rn(x, inv));
 }
 
-template <int FMT> __device__ __noinline__ uint4 encode16_careful(const uint32_t (&w)[8], float inv)
+// Rare path, kept out of line and fed by value so that the common path keeps its data in registers.
+template <int FMT> __device__ __noinline__ uint4 encode16_careful(uint4 lo, uint4 hi, float inv)
 {
+    const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
     uint32_t c[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -84,212 +218,393 @@ template <int FMT> __device__ __noinline__ uint4 encode16_careful(const uint32_t
     return make_uint4(c[0], c[1], c[2], c[3]);
 }
 
-// max |bits| over the finite elements only
-__device__ __noinline__ uint32_t absmax_bits16_finite(const uint32_t (&w)[8])
+// max |bits| over the finite elements only (rare path, by value)
+__device__ __noinline__ uint32_t absmax16_finite(uint4 lo, uint4 hi)
 {
+    const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
     uint32_t m = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        uint32_t lo = w[i] & 0x7FFFu, hi = (w[i] >> 16) & 0x7FFFu;
-        if (lo < 0x7F80u) m = max(m, lo);
-        if (hi < 0x7F80u) m = max(m, hi);
+        uint32_t l = w[i] & 0x7FFFu, h = (w[i] >> 16) & 0x7FFFu;
+        if (l < 0x7F80u) m = max(m, l);
+        if (h < 0x7F80u) m = max(m, h);
     }
     return m;
 }
 
-__device__ __forceinline__ float sumsq16(const uint32_t (&w)[8])
+#define HILORE_LO4(w) make_uint4((w)[0], (w)[1], (w)[2], (w)[3])
+#define HILORE_HI4(w) make_uint4((w)[4], (w)[5], (w)[6], (w)[7])
+
+// One pass over a chunk: unpack each bf16 pair once, feed it to the sum of squares (SUMS) and to the
+// scaled conversion (CODES).  Elements must be finite (BLK) / at most 464 in magnitude (RAW).
+template <int FMT, bool CODES, bool SUMS>
+__device__ __forceinline__ void chunk_pass(const uint32_t (&w)[8], float inv, uint4 &codes, float &sumsq)
 {
-    float a = 0.0f, b = 0.0f;
+    const uint64_t inv2 = f32x2_pack(inv, inv);
+    uint64_t acc = 0; // {0.0f, 0.0f}
+    uint32_t h[8];    // two codes per word
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        float lo = bf16_lo(w[i]), hi = bf16_hi(w[i]);
-        a = fmaf(lo, lo, a);
-        b = fmaf(hi, hi, b);
+        uint64_t x = f32x2_pack(bf16_lo(w[i]), bf16_hi(w[i]));
+        if (SUMS)
+            acc = f32x2_fma(x, x, acc);
+        if (CODES) {
+            if (FMT != HILORE_FMT_E4M3FN_RAW)
+                x = f32x2_mul(x, inv2); // fl32(x * inv), each lane rounded to nearest even
+            float lo, hi;
+            f32x2_unpack(x, lo, hi);
+            if (FMT == HILORE_FMT_INT8_BLK)
+                h[i] = int8_code(lo) | (int8_code(hi) << 8);
+            else
+                h[i] = cvt_e4m3x2(hi, lo);
+        }
     }
-    return a + b;
+    if (CODES)
+        codes = make_uint4(__byte_perm(h[0], h[1], 0x5410), __byte_perm(h[2], h[3], 0x5410),
+                           __byte_perm(h[4], h[5], 0x5410), __byte_perm(h[6], h[7], 0x5410));
+    if (SUMS) {
+        float lo, hi;
+        f32x2_unpack(acc, lo, hi);
+        sumsq = lo + hi;
+    }
 }
 
-struct RowGeom {
-    int64_t cols, ld;   // elements
-    uint32_t cpr;       // 16-element chunks per row
-    uint32_t nb;        // 64-element blocks per row
-    uint32_t magic;     // ceil(2^32 / cpr): exact division of chunk indices < 2^16 by cpr
-    int rows_per_batch; // rows swept between two row reductions
-};
-
-__device__ __forceinline__ RowGeom make_geom(int64_t cols, int64_t ld)
+// Everything a thread does with the two chunks it holds.  All 32 lanes must call this together
+// (xor-shuffles inside).  The four lanes of a quad hold one 64-element block per chunk.
+//   CODES: the two IEEE divisions of a block (s = amax / Q, inv = Q / amax) are spread over the quad:
+//          lanes 0 / 1 compute s / inv of chunk 0's block, lanes 2 / 3 those of chunk 1's block -- one
+//          division per thread instead of four.  `s_store` is the scale of chunk 0's block in lanes with
+//          (lane & 3) == 0 and of chunk 1's block in lanes with (lane & 3) == 2.
+//   SUMS:  `bsum` is the block sum of squares of chunk 0's block in even lanes, of chunk 1's in odd lanes.
+template <int FMT, bool CODES, bool SUMS>
+__device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint32_t (&w1)[8], int lane, uint4 &c0,
+                                             uint4 &c1, float &s_store, float &bsum)
 {
-    RowGeom g;
-    g.cols = cols;
-    g.ld = ld;
-    g.cpr = (uint32_t)(cols >> 4);
-    g.nb = (uint32_t)(cols >> 6);
-    g.magic = (uint32_t)((0x100000000ull + g.cpr - 1) / g.cpr);
-    g.rows_per_batch = max(1, kBlockSumSlots / (int)g.nb);
-    return g;
-}
-
-// Element offset of chunk c (within a batch that starts at row `row0`) in a [rows, ld] tensor.
-__device__ __forceinline__ int64_t chunk_offset(const RowGeom &g, int64_t row0, uint32_t c, int64_t ld)
-{
-    if (ld == g.cols)
-        return row0 * ld + (int64_t)c * 16;
-    uint32_t r = __umulhi(c, g.magic);
-    uint32_t cc = c - r * g.cpr;
-    return (row0 + r) * ld + (int64_t)cc * 16;
-}
-
-// Compress (CODES) and / or collect the token RMS of rows [r0, r1) of one unit.
-template <int FMT, bool CODES, int UNR>
-__device__ void compress_rows(const hilore_unit &u, int64_t r0, int64_t r1, float *sm_blocksum)
-{
-    const RowGeom g = make_geom(u.cols, u.ld);
-    const uint16_t *x = static_cast<const uint16_t *>(u.x);
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const uint32_t quad_mask = 0xFu << (lane & 28);
-    const bool want_rms = (u.row_rms != nullptr);
     constexpr float Q = QMax<FMT>::value;
-
-    for (int64_t rb0 = r0; rb0 < r1; rb0 += g.rows_per_batch) {
-        const int rb = (int)min((int64_t)g.rows_per_batch, r1 - rb0);
-        const uint32_t n = (uint32_t)rb * g.cpr; // chunks of this batch, <= 4 * kBlockSumSlots
-        for (uint32_t base = 0; base < n; base += kCodecThreads * UNR) {
-            uint32_t w[UNR][8];
-            bool valid[UNR];
-#pragma unroll
-            for (int j = 0; j < UNR; ++j) {
-                const uint32_t c = base + j * kCodecThreads + tid;
-                valid[j] = c < n;
-                if (valid[j]) {
-                    ld_global_256(x + chunk_offset(g, rb0, c, g.ld), w[j]);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) w[j][i] = 0;
-                }
+    float inv0 = 1.0f, inv1 = 1.0f;
+    bool careful0 = false, careful1 = false;
+    s_store = 1.0f;
+    if (CODES) {
+        uint32_t m0 = absmax16(w0), m1 = absmax16(w1);
+        if (FMT == HILORE_FMT_E4M3FN_RAW) {
+            careful0 = m0 > 0x43E8u;
+            careful1 = m1 > 0x43E8u;
+        } else {
+            uint32_t mp = m0 | (m1 << 16); // both blocks' maxima ride in one register through the quad
+            mp = maxnan_bf16x2(mp, __shfl_xor_sync(0xFFFFFFFFu, mp, 1));
+            mp = maxnan_bf16x2(mp, __shfl_xor_sync(0xFFFFFFFFu, mp, 2));
+            m0 = mp & 0xFFFFu;
+            m1 = mp >> 16;
+            careful0 = careful1 = (m0 >= 0x7F80u) || (m1 >= 0x7F80u); // uniform over the quad
+            if (careful0) { // Inf or NaN in one of the two blocks: absmax over the finite elements only
+                const uint32_t quad_mask = 0xFu << (lane & 28);
+                uint32_t f0 = absmax16_finite(HILORE_LO4(w0), HILORE_HI4(w0));
+                uint32_t f1 = absmax16_finite(HILORE_LO4(w1), HILORE_HI4(w1));
+                f0 = max(f0, __shfl_xor_sync(quad_mask, f0, 1));
+                f1 = max(f1, __shfl_xor_sync(quad_mask, f1, 1));
+                m0 = max(f0, __shfl_xor_sync(quad_mask, f0, 2));
+                m1 = max(f1, __shfl_xor_sync(quad_mask, f1, 2));
             }
+            const int q = lane & 3;
+            const float a = __uint_as_float(((q & 2) ? m1 : m0) << 16);
+            const float r = __fdiv_rn((q & 1) ? Q : a, (q & 1) ? a : Q); // s in even lanes, inv in odd lanes
+            const bool unit0 = m0 <= UnitScaleBelow<FMT>::value, unit1 = m1 <= UnitScaleBelow<FMT>::value;
+            inv0 = __shfl_sync(0xFFFFFFFFu, r, (lane & 28) | 1);
+            inv1 = __shfl_sync(0xFFFFFFFFu, r, (lane & 28) | 3);
+            inv0 = unit0 ? 1.0f : inv0;
+            inv1 = unit1 ? 1.0f : inv1;
+            s_store = ((q & 2) ? unit1 : unit0) ? 1.0f : r;
+        }
+    }
+    float ss0 = 0.0f, ss1 = 0.0f;
+    chunk_pass<FMT, CODES, SUMS>(w0, inv0, c0, ss0);
+    chunk_pass<FMT, CODES, SUMS>(w1, inv1, c1, ss1);
+    if (CODES) {
+        if (careful0) c0 = encode16_careful<FMT>(HILORE_LO4(w0), HILORE_HI4(w0), inv0);
+        if (careful1) c1 = encode16_careful<FMT>(HILORE_LO4(w1), HILORE_HI4(w1), inv1);
+    }
+    if (SUMS) { // quad reduction of both blocks' sums with two shuffles
+        const bool odd = lane & 1;
+        float keep = odd ? ss1 : ss0;
+        keep += __shfl_xor_sync(0xFFFFFFFFu, odd ? ss0 : ss1, 1);
+        keep += __shfl_xor_sync(0xFFFFFFFFu, keep, 2);
+        bsum = keep;
+    }
+}
+
+__device__ __forceinline__ void zero8(uint32_t (&w)[8])
+{
 #pragma unroll
-            for (int j = 0; j < UNR; ++j) {
-                const uint32_t c = base + j * kCodecThreads + tid;
-                // n is a multiple of 4 and quads start at multiples of 4: a quad is valid as a whole
+    for (int i = 0; i < 8; ++i) w[i] = 0;
+}
+
+// Compress (CODES) and / or collect the token RMS (SUMS) of rows [r0, r1) of one unit.
+template <int FMT, bool CODES, bool SUMS>
+__device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, uint8_t *__restrict__ codes,
+                                              float *__restrict__ scales, float *__restrict__ row_rms, int64_t cols,
+                                              int64_t ld, int64_t r0, int64_t r1, float *sm_blocksum, int prefetch)
+{
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, q = lane & 3;
+    const uint32_t nb = (uint32_t)(cols >> 6), cpr = (uint32_t)(cols >> 4);
+    const int rows_per_batch = max(1, kBlockSumSlots / (int)nb);
+    const uint32_t magic = (uint32_t)((0x100000000ull + cpr - 1) / cpr); // chunk index (< 2^16) / cpr, exactly
+    const float inv_cols = 1.0f / (float)cols;
+    const bool contig = ld == cols;
+
+    for (int64_t rb0 = r0; rb0 < r1; rb0 += rows_per_batch) {
+        const int rb = (int)min((int64_t)rows_per_batch, r1 - rb0);
+        const uint32_t n = (uint32_t)rb * cpr; // chunks of this batch (a multiple of 4), <= 4 * kBlockSumSlots
+        const uint16_t *xb = x + rb0 * ld;
+        uint8_t *cb_ = codes + rb0 * cols;
+        float *sb = scales + rb0 * (int64_t)nb;
+        uint32_t base = 0;
+        if (contig) { // whole iterations: no predicates, pointer increments only
+            const uint16_t *xp = xb + (size_t)tid * 16;
+            uint8_t *cp = cb_ + (size_t)tid * 16;
+            float *sp = sb + (tid >> 2);
+            float *bp = sm_blocksum + (tid >> 2);
+            // One iteration of the CTA reads 16 KB contiguously.  An elected thread keeps the copy engine
+            // `prefetch` iterations ahead, pulling those 16 KB pieces from HBM into L2, so that the warps'
+            // own loads find their data in L2 and HBM traffic no longer waits for warp progress.
+            constexpr uint32_t kIterBytes = 2 * kCodecThreads * 32;
+            const uint32_t full_iters = n / (2 * kCodecThreads);
+            const uint8_t *pf = reinterpret_cast<const uint8_t *>(xb);
+            if (tid == 0)
+                for (uint32_t k = 0; k < (uint32_t)prefetch && k < full_iters; ++k) prefetch_l2_bulk(pf + (size_t)k * kIterBytes, kIterBytes);
+            uint32_t iter = 0;
+            for (; base + 2 * kCodecThreads <= n; base += 2 * kCodecThreads, ++iter) {
+                if (tid == 0 && prefetch > 0 && iter + prefetch < full_iters)
+                    prefetch_l2_bulk(pf + (size_t)(iter + prefetch) * kIterBytes, kIterBytes);
+                uint32_t wa[8], wb[8];
+                ld_global_256(xp, wa);
+                ld_global_256(xp + kCodecThreads * 16, wb);
+                uint4 qa, qb;
+                float s, ss;
+                process_pair<FMT, CODES, SUMS>(wa, wb, lane, qa, qb, s, ss);
                 if (CODES) {
-                    uint32_t mm = absmax_bits16(w[j]);
-                    float s = 1.0f, inv = 1.0f;
-                    bool careful;
-                    if (FMT == HILORE_FMT_E4M3FN_RAW) {
-                        careful = mm > 0x43E8u;
-                    } else {
-                        mm = max(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, 1));
-                        mm = max(mm, __shfl_xor_sync(0xFFFFFFFFu, mm, 2));
-                        careful = mm >= 0x7F80u;
-                        if (careful) { // the block holds Inf or NaN: absmax over its finite elements
-                            mm = absmax_bits16_finite(w[j]);
-                            mm = max(mm, __shfl_xor_sync(quad_mask, mm, 1));
-                            mm = max(mm, __shfl_xor_sync(quad_mask, mm, 2));
-                        }
-                        if (mm != 0) {
-                            const float amax = __uint_as_float(mm << 16);
-                            s = __fdiv_rn(amax, Q);
-                            inv = __fdiv_rn(Q, amax);
-                            if (isinf(inv)) {
-                                s = 1.0f;
-                                inv = 1.0f;
-                            }
-                        }
-                    }
-                    if (valid[j]) {
-                        const uint4 codes = careful ? encode16_careful<FMT>(w[j], inv) : encode16_fast<FMT>(w[j], inv);
-                        const int64_t flat = rb0 * g.cols + (int64_t)c * 16;
-                        *reinterpret_cast<uint4 *>(u.codes + flat) = codes;
-                        if (FMT != HILORE_FMT_E4M3FN_RAW && (lane & 3) == 0)
-                            u.scales[rb0 * g.nb + (c >> 2)] = s;
+                    *reinterpret_cast<uint4 *>(cp) = qa;
+                    *reinterpret_cast<uint4 *>(cp + kCodecThreads * 16) = qb;
+                    if (FMT != HILORE_FMT_E4M3FN_RAW) {
+                        if (q == 0) sp[0] = s;
+                        if (q == 2) sp[kCodecThreads / 4] = s;
                     }
                 }
-                if (want_rms) {
-                    float ss = sumsq16(w[j]);
-                    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
-                    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
-                    if (valid[j] && (lane & 3) == 0)
-                        sm_blocksum[c >> 2] = ss;
+                if (SUMS) {
+                    if (q == 0) bp[0] = ss;
+                    if (q == 1) bp[kCodecThreads / 4] = ss;
                 }
+                xp += 2 * kCodecThreads * 16;
+                cp += 2 * kCodecThreads * 16;
+                sp += 2 * kCodecThreads / 4;
+                bp += 2 * kCodecThreads / 4;
             }
         }
-        if (want_rms) {
+        for (; base < n; base += 2 * kCodecThreads) { // ragged end of a batch, or rows with a leading dimension
+            const uint32_t ca = base + tid, cb = ca + kCodecThreads;
+            const bool va = ca < n, vb = cb < n; // quads are valid as a whole (n is a multiple of 4)
+            uint32_t wa[8], wb[8];
+            zero8(wa);
+            zero8(wb);
+            if (va) {
+                const uint32_t r = __umulhi(ca, magic);
+                ld_global_256(xb + (int64_t)r * ld + (int64_t)(ca - r * cpr) * 16, wa);
+            }
+            if (vb) {
+                const uint32_t r = __umulhi(cb, magic);
+                ld_global_256(xb + (int64_t)r * ld + (int64_t)(cb - r * cpr) * 16, wb);
+            }
+            uint4 qa, qb;
+            float s, ss;
+            process_pair<FMT, CODES, SUMS>(wa, wb, lane, qa, qb, s, ss);
+            if (CODES) {
+                if (va) *reinterpret_cast<uint4 *>(cb_ + (size_t)ca * 16) = qa;
+                if (vb) *reinterpret_cast<uint4 *>(cb_ + (size_t)cb * 16) = qb;
+                if (FMT != HILORE_FMT_E4M3FN_RAW) {
+                    if (q == 0 && va) sb[ca >> 2] = s;
+                    if (q == 2 && vb) sb[cb >> 2] = s;
+                }
+            }
+            if (SUMS) {
+                if (q == 0 && va) sm_blocksum[ca >> 2] = ss;
+                if (q == 1 && vb) sm_blocksum[cb >> 2] = ss;
+            }
+        }
+        if (SUMS) {
             __syncthreads();
             for (int r = wid; r < rb; r += kCodecThreads / 32) {
                 double acc = 0.0;
-                for (uint32_t b = lane; b < g.nb; b += 32)
-                    acc += (double)sm_blocksum[(uint32_t)r * g.nb + b];
+                for (uint32_t b = lane; b < nb; b += 32)
+                    acc += (double)sm_blocksum[(uint32_t)r * nb + b];
                 acc = warp_sum(acc);
                 if (lane == 0)
-                    u.row_rms[rb0 + r] = (float)sqrt(acc / (double)g.cols);
+                    row_rms[rb0 + r] = sqrtf((float)acc * inv_cols);
             }
             __syncthreads();
         }
     }
 }
 
-// Decode rows [r0, r1) of one unit into u.out.
-template <int FMT, int UNR> __device__ void recover_rows(const hilore_unit &u, int64_t r0, int64_t r1)
+// Sixteen codes -> sixteen bf16 (eight words).
+template <int FMT> __device__ __forceinline__ void decode16(const uint4 cd, float s, uint32_t (&o)[8])
 {
-    const RowGeom g = make_geom(u.cols, u.ld);
-    uint16_t *out = static_cast<uint16_t *>(u.out);
+    const uint64_t s2 = f32x2_pack(s, s);
+    const uint32_t cw[4] = {cd.x, cd.y, cd.z, cd.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            const uint32_t two = p ? (cw[i] >> 16) : (cw[i] & 0xFFFFu); // two codes
+            float f0, f1;
+            if (FMT == HILORE_FMT_INT8_BLK) {
+                const int b0 = (int)(int8_t)(two & 0xFF), b1 = (int)(int8_t)(two >> 8);
+                const float qnan = __uint_as_float(0x7FC00000u);
+                f0 = (b0 == -128) ? qnan : (float)b0;
+                f1 = (b1 == -128) ? qnan : (float)b1;
+            } else {
+                const uint32_t hh = cvt_e4m3x2_to_f16x2(two);
+                f0 = f16_lo_to_f32(hh);
+                f1 = f16_hi_to_f32(hh);
+            }
+            if (FMT != HILORE_FMT_E4M3FN_RAW) {
+                const uint64_t y = f32x2_mul(f32x2_pack(f0, f1), s2); // fl32(value * s) per lane
+                f32x2_unpack(y, f0, f1);
+            }
+            o[2 * i + p] = cvt_bf16x2(f1, f0);
+        }
+    }
+}
+
+// Decode rows [r0, r1) of one unit.
+template <int FMT>
+__device__ __forceinline__ void recover_rows(const uint8_t *__restrict__ codes, const float *__restrict__ scales,
+                                             uint16_t *__restrict__ out, int64_t cols, int64_t ld, int64_t r0, int64_t r1,
+                                             int prefetch)
+{
+    constexpr int UNR = 4;
     const int tid = threadIdx.x;
-    for (int64_t rb0 = r0; rb0 < r1; rb0 += g.rows_per_batch) {
-        const int rb = (int)min((int64_t)g.rows_per_batch, r1 - rb0);
-        const uint32_t n = (uint32_t)rb * g.cpr;
-        for (uint32_t base = 0; base < n; base += kCodecThreads * UNR) {
+    const int64_t nb = cols >> 6, cpr = cols >> 4;
+    const int64_t n = (r1 - r0) * cpr; // chunks of this CTA's rows
+    const uint8_t *cb_ = codes + r0 * cols;
+    const float *sb = scales + r0 * nb;
+    int64_t base = 0;
+    if (ld == cols) {
+        const uint8_t *cp = cb_ + (size_t)tid * 16;
+        const float *sp = sb + (tid >> 2);
+        uint16_t *op = out + r0 * ld + (size_t)tid * 16;
+        constexpr uint32_t kIterBytes = UNR * kCodecThreads * 16; // codes read per iteration of the CTA
+        const int64_t full_iters = n / (UNR * kCodecThreads);
+        if (tid == 0)
+            for (int64_t k = 0; k < prefetch && k < full_iters; ++k) prefetch_l2_bulk(cb_ + k * kIterBytes, kIterBytes);
+        int64_t iter = 0;
+        for (; base + UNR * kCodecThreads <= n; base += UNR * kCodecThreads, ++iter) {
+            if (tid == 0 && prefetch > 0 && iter + prefetch < full_iters)
+                prefetch_l2_bulk(cb_ + (iter + prefetch) * kIterBytes, kIterBytes);
             uint4 cd[UNR];
             float s[UNR];
-            bool valid[UNR];
 #pragma unroll
             for (int j = 0; j < UNR; ++j) {
-                const uint32_t c = base + j * kCodecThreads + tid;
-                valid[j] = c < n;
-                s[j] = 1.0f;
-                cd[j] = make_uint4(0, 0, 0, 0);
-                if (valid[j]) {
-                    cd[j] = ld_global_128_stream(u.codes + rb0 * g.cols + (int64_t)c * 16);
-                    if (FMT != HILORE_FMT_E4M3FN_RAW)
-                        s[j] = __ldg(u.scales + rb0 * g.nb + (c >> 2));
-                }
+                cd[j] = ld_global_128_stream(cp + (size_t)j * kCodecThreads * 16);
+                s[j] = (FMT != HILORE_FMT_E4M3FN_RAW) ? __ldg(sp + j * (kCodecThreads / 4)) : 1.0f;
             }
 #pragma unroll
             for (int j = 0; j < UNR; ++j) {
-                if (!valid[j])
-                    continue;
-                const uint32_t c = base + j * kCodecThreads + tid;
-                const uint32_t cw[4] = {cd[j].x, cd[j].y, cd[j].z, cd[j].w};
                 uint32_t o[8];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float f0, f1, f2, f3;
-                    if (FMT == HILORE_FMT_INT8_BLK) {
-                        const int b0 = (int)(int8_t)(cw[i] & 0xFF), b1 = (int)(int8_t)((cw[i] >> 8) & 0xFF);
-                        const int b2 = (int)(int8_t)((cw[i] >> 16) & 0xFF), b3 = (int)(int8_t)(cw[i] >> 24);
-                        const float qnan = __uint_as_float(0x7FC00000u);
-                        f0 = (b0 == -128) ? qnan : (float)b0;
-                        f1 = (b1 == -128) ? qnan : (float)b1;
-                        f2 = (b2 == -128) ? qnan : (float)b2;
-                        f3 = (b3 == -128) ? qnan : (float)b3;
-                    } else {
-                        const uint32_t h01 = cvt_e4m3x2_to_f16x2(cw[i] & 0xFFFFu);
-                        const uint32_t h23 = cvt_e4m3x2_to_f16x2(cw[i] >> 16);
-                        f0 = f16_lo_to_f32(h01);
-                        f1 = f16_hi_to_f32(h01);
-                        f2 = f16_lo_to_f32(h23);
-                        f3 = f16_hi_to_f32(h23);
-                    }
-                    if (FMT != HILORE_FMT_E4M3FN_RAW) {
-                        f0 = __fmul_rn(f0, s[j]);
-                        f1 = __fmul_rn(f1, s[j]);
-                        f2 = __fmul_rn(f2, s[j]);
-                        f3 = __fmul_rn(f3, s[j]);
-                    }
-                    o[2 * i] = cvt_bf16x2(f1, f0);
-                    o[2 * i + 1] = cvt_bf16x2(f3, f2);
-                }
-                st_global_256(out + chunk_offset(g, rb0, c, g.ld), o);
+                decode16<FMT>(cd[j], s[j], o);
+                st_global_256(op + (size_t)j * kCodecThreads * 16, o);
             }
+            cp += UNR * kCodecThreads * 16;
+            sp += UNR * kCodecThreads / 4;
+            op += UNR * kCodecThreads * 16;
+        }
+    }
+    for (; base < n; base += kCodecThreads) {
+        const int64_t c = base + tid;
+        if (c < n) {
+            const uint4 cd = ld_global_128_stream(cb_ + c * 16);
+            const float s = (FMT != HILORE_FMT_E4M3FN_RAW) ? __ldg(sb + (c >> 2)) : 1.0f;
+            uint32_t o[8];
+            decode16<FMT>(cd, s, o);
+            const int64_t r = c / cpr;
+            st_global_256(out + (r0 + r) * ld + (c - r * cpr) * 16, o);
+        }
+    }
+}
+
+
+// ---- bulk stores (copy engine): shared memory -> global, tracked in per-thread groups ----
+__device__ __forceinline__ void bulk_s2g(void *dst_gmem, const void *src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst_gmem),
+                 "r"((uint32_t)__cvta_generic_to_shared(src_smem)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all but the newest N bulk-store groups of this thread have finished reading shared memory
+template <int N> __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// make this thread's shared-memory writes visible to the copy engine
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+constexpr int kRecoverTileChunks = 2 * kCodecThreads;        // 512 chunks = 8192 elements per tile
+constexpr int kRecoverTileBytes = kRecoverTileChunks * 32;   // 16 KB of bf16
+constexpr int kRecoverStageBytes = 2 * kRecoverTileBytes;    // two tiles in shared memory
+
+// Decode rows [r0, r1) of a contiguous unit (ld == cols).  The pass writes twice what it reads, and HBM
+// takes writes best in large contiguous bursts: each tile of 8192 reconstructed values is assembled in
+// shared memory and sent with one 16 KB bulk store while the threads work on the next tile (two buffers;
+// a buffer is refilled only after the store that read it has finished reading).
+// `tile` counts this CTA's tiles across calls, so the two buffers keep alternating from unit to unit.
+template <int FMT>
+__device__ __forceinline__ void recover_rows_bulk(const uint8_t *__restrict__ codes, const float *__restrict__ scales,
+                                                  uint16_t *__restrict__ out, int64_t cols, int64_t r0, int64_t r1,
+                                                  uint8_t *sm_out, uint32_t &tile, int prefetch)
+{
+    const int tid = threadIdx.x;
+    const int64_t nb = cols >> 6, cpr = cols >> 4;
+    const int64_t n = (r1 - r0) * cpr; // chunks of this CTA's rows
+    const uint8_t *cb_ = codes + r0 * cols;
+    const float *sb = scales + r0 * nb;
+    uint8_t *ob = reinterpret_cast<uint8_t *>(out + r0 * cols);
+    const int64_t ntiles = (n + kRecoverTileChunks - 1) / kRecoverTileChunks;
+    if (tid == 0)
+        for (int64_t k = 0; k < prefetch && k < ntiles; ++k)
+            prefetch_l2_bulk(cb_ + k * kRecoverTileChunks * 16, (uint32_t)min((int64_t)kRecoverTileChunks, n - k * kRecoverTileChunks) * 16);
+    for (int64_t t = 0; t < ntiles; ++t, ++tile) {
+        const int64_t base = t * kRecoverTileChunks;
+        if (tid == 0 && prefetch > 0 && t + prefetch < ntiles)
+            prefetch_l2_bulk(cb_ + (t + prefetch) * kRecoverTileChunks * 16,
+                             (uint32_t)min((int64_t)kRecoverTileChunks, n - (t + prefetch) * kRecoverTileChunks) * 16);
+        const int64_t ca = base + tid, cb = ca + kCodecThreads;
+        const bool va = ca < n, vb = cb < n;
+        uint4 cda = make_uint4(0, 0, 0, 0), cdb = cda;
+        float sa = 1.0f, sb_ = 1.0f;
+        if (va) {
+            cda = ld_global_128_stream(cb_ + ca * 16);
+            if (FMT != HILORE_FMT_E4M3FN_RAW) sa = __ldg(sb + (ca >> 2));
+        }
+        if (vb) {
+            cdb = ld_global_128_stream(cb_ + cb * 16);
+            if (FMT != HILORE_FMT_E4M3FN_RAW) sb_ = __ldg(sb + (cb >> 2));
+        }
+        uint32_t oa[8], ob2[8];
+        decode16<FMT>(cda, sa, oa);
+        decode16<FMT>(cdb, sb_, ob2);
+        uint8_t *buf = sm_out + (tile & 1u) * kRecoverTileBytes;
+        if (tid == 0)
+            bulk_wait_read<1>(); // the store issued two tiles ago (same buffer) has finished reading it
+        __syncthreads();
+        uint4 *pa = reinterpret_cast<uint4 *>(buf + (size_t)tid * 32);
+        uint4 *pb = reinterpret_cast<uint4 *>(buf + (size_t)(tid + kCodecThreads) * 32);
+        pa[0] = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+        pa[1] = make_uint4(oa[4], oa[5], oa[6], oa[7]);
+        pb[0] = make_uint4(ob2[0], ob2[1], ob2[2], ob2[3]);
+        pb[1] = make_uint4(ob2[4], ob2[5], ob2[6], ob2[7]);
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            const uint32_t bytes = (uint32_t)min((int64_t)kRecoverTileChunks, n - base) * 32u;
+            bulk_s2g(ob + base * 32, buf, bytes);
+            bulk_commit();
         }
     }
 }

@@ -39,6 +39,13 @@ __device__ __forceinline__ uint4 ld_global_128_stream(const void *p)
     return v;
 }
 
+// Ask the copy engine to pull `bytes` (a multiple of 16, 16-byte aligned) from HBM into L2, no register or
+// shared-memory destination: the later plain loads of this range then hit L2.
+__device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // ---- packed conversions ----
 // Two fp32 -> two E4M3FN codes, round to nearest even, saturating at +-448; `lo` lands in the low byte.
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo)
@@ -81,20 +88,35 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float hi, float lo)
     return r;
 }
 
+// ---- packed fp32 pairs (sm_100: one instruction per two fp32 lanes, each lane rounded as IEEE RN) ----
+__device__ __forceinline__ uint64_t f32x2_pack(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+
+__device__ __forceinline__ void f32x2_unpack(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
+__device__ __forceinline__ uint64_t f32x2_mul(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
+__device__ __forceinline__ uint64_t f32x2_fma(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
-
-// max over the sixteen |bf16| bit patterns held in w[0..7] (as unsigned 16-bit integers, so that
-// Inf and NaN patterns (>= 0x7F80) compare above every finite value).
-__device__ __forceinline__ uint32_t absmax_bits16(const uint32_t (&w)[8])
-{
-    const uint32_t M = 0x7FFF7FFFu;
-    uint32_t a = __vimax3_u16x2(w[0] & M, w[1] & M, w[2] & M);
-    uint32_t b = __vimax3_u16x2(w[3] & M, w[4] & M, w[5] & M);
-    uint32_t c = __vimax3_u16x2(w[6] & M, w[7] & M, a);
-    uint32_t m = __vmaxu2(b, c);
-    return max(m & 0xFFFFu, m >> 16);
-}
 
 __device__ __forceinline__ double warp_sum(double v)
 {
@@ -114,9 +136,6 @@ __device__ __forceinline__ float warp_sum(float v)
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-struct DeviceInfo {
-    int sms;
-};
 // Number of SMs of the current device (queried each call; the library keeps no state).
 inline int sm_count()
 {

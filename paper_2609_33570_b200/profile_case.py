@@ -12,7 +12,8 @@ import torch
 from . import api, synth
 
 
-def codec_case(rows: int, cols: int, fmt: int, reps: int, units: int):
+def codec_case(rows: int, cols: int, fmt: int, reps: int, units: int, rms: bool = True, codes_on: bool = True,
+               recover: bool = True):
     gen = torch.Generator(device="cuda")
     gen.manual_seed(0)
     block = 0 if fmt == api.FMT_E4M3FN_RAW else 64
@@ -20,11 +21,12 @@ def codec_case(rows: int, cols: int, fmt: int, reps: int, units: int):
     codes = [torch.empty((rows, cols), dtype=torch.uint8, device="cuda") for _ in range(units)]
     scales = [torch.empty((rows, max(cols // 64, 1)), dtype=torch.float32, device="cuda") for _ in range(units)]
     outs = [torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda") for _ in range(units)]
-    rms = torch.empty((units, rows), dtype=torch.float32, device="cuda")
+    rms_buf = torch.empty((units, rows), dtype=torch.float32, device="cuda")
     for _ in range(reps):
         for i in range(units):
-            api.hilore_compress(xs[i], rows, cols, cols, fmt, block, codes[i], scales[i] if block else None, rms[i])
-        for i in range(units):
+            api.hilore_compress(xs[i], rows, cols, cols, fmt, block, codes[i] if codes_on else None,
+                                scales[i] if (block and codes_on) else None, rms_buf[i] if (rms or not codes_on) else None)
+        for i in range(units if recover else 0):
             api.hilore_recover(codes[i], scales[i] if block else None, rows, cols, fmt, block, outs[i], cols)
     torch.cuda.synchronize()
 
@@ -53,9 +55,13 @@ def main():
     ap.add_argument("--units", type=int, default=2)
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--log2-slots", type=int, default=24)
+    ap.add_argument("--no-rms", action="store_true", help="compress without the fused token RMS")
+    ap.add_argument("--stats-only", action="store_true", help="token RMS only, no codes")
+    ap.add_argument("--no-recover", action="store_true")
     a = ap.parse_args()
     if a.kernel == "codec":
-        codec_case(a.rows, a.cols, a.fmt, a.reps, a.units)
+        codec_case(a.rows, a.cols, a.fmt, a.reps, a.units, rms=not a.no_rms, codes_on=not a.stats_only,
+                   recover=not a.no_recover)
     else:
         coeffs_case(a.log2_slots, a.reps)
     print("done")

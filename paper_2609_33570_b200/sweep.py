@@ -1,0 +1,103 @@
+"""Bandwidth sweep of the single-unit entry points (`python -m paper_2609_33570_b200.sweep`).
+
+Units [rows, cols] bf16 of 1 MiB ... 4 GiB (row width 4096 by default), compress then recover, and the
+coefficient kernel over 2^16 ... 2^24 slots at G = 16.  Each point is timed with CUDA events over `reps`
+calls that rotate through a pool of distinct buffers larger than L2, so the numbers are HBM numbers.
+Prints one JSON line per point.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import api, synth
+
+L2_BYTES = 126 << 20
+
+
+def _time(fn_list, reps):
+    for f in fn_list[: min(len(fn_list), 3)]:
+        f()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(reps):
+        fn_list[i % len(fn_list)]()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def codec_point(rows, cols, fmt, reps, with_rms=True, max_pool_bytes=6 << 30):
+    block = 0 if fmt == api.FMT_E4M3FN_RAW else 64
+    unit_bytes = rows * cols * 2
+    pool = max(1, min(8, -(-3 * L2_BYTES // unit_bytes)))          # enough distinct units to defeat L2
+    pool = max(1, min(pool, max_pool_bytes // (unit_bytes * 2 + rows * cols)))
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(0)
+    base = synth.activation_unit_device(gen, min(rows, 4096), cols)
+    xs = [base.repeat(-(-rows // base.shape[0]), 1)[:rows].contiguous() for _ in range(pool)]
+    codes = [torch.empty((rows, cols), dtype=torch.uint8, device="cuda") for _ in range(pool)]
+    scales = [torch.empty((rows, max(cols // 64, 1)), dtype=torch.float32, device="cuda") for _ in range(pool)]
+    outs = [torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda") for _ in range(pool)]
+    rms = torch.empty(rows, dtype=torch.float32, device="cuda")
+    comp = [lambda i=i: api.hilore_compress(xs[i], rows, cols, cols, fmt, block, codes[i], scales[i] if block else None,
+                                            rms if with_rms else None) for i in range(pool)]
+    rec = [lambda i=i: api.hilore_recover(codes[i], scales[i] if block else None, rows, cols, fmt, block, outs[i], cols)
+           for i in range(pool)]
+    n = rows * cols
+    nbytes = 3 * n + (4 * n // 64 if block else 0)
+    tc, tr = _time(comp, reps), _time(rec, reps)
+    return {"kernel": "codec", "rows": rows, "cols": cols, "fmt": fmt, "unit_mib": unit_bytes / 2 ** 20, "pool": pool,
+            "compress_us": tc * 1e3, "compress_gbs": (nbytes + (4 * rows if with_rms else 0)) / tc / 1e6,
+            "recover_us": tr * 1e3, "recover_gbs": nbytes / tr / 1e6}
+
+
+def coeffs_point(log2_slots, reps, G=16, T=1024):
+    n_resp = max(G, (1 << log2_slots) // T)
+    slots = n_resp * T
+    pool = max(1, min(8, -(-3 * L2_BYTES // (slots * 13))))
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1)
+    lp = [torch.randn((n_resp, T), generator=gen, device="cuda") * 0.5 - 1.5 for _ in range(pool)]
+    lo = [x + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.05 for x in lp]
+    mask = torch.ones((n_resp, T), dtype=torch.uint8, device="cuda")
+    rewards = (torch.rand(n_resp, generator=gen, device="cuda") < 0.5).float()
+    omega = [torch.empty_like(x) for x in lp]
+    fns = [lambda i=i: api.hilore_grpo_coeffs(rewards, n_resp, G, 0, n_resp, T, lp[i], lo[i], None, mask, slots, None, 0.2,
+                                              0.0, 1e-6, None, omega[i], None, None) for i in range(pool)]
+    t = _time(fns, reps)
+    return {"kernel": "grpo_coeffs", "slots": slots, "pool": pool, "us": t * 1e3, "tokens_per_s": slots / t * 1e3,
+            "gbs": 13 * slots / t / 1e6}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--cols", type=int, default=4096)
+    ap.add_argument("--min-log2-rows", type=int, default=7)
+    ap.add_argument("--max-log2-rows", type=int, default=19)
+    ap.add_argument("--fmts", type=int, nargs="*", default=[api.FMT_E4M3FN_RAW, api.FMT_E4M3FN_BLK])
+    ap.add_argument("--shapes", type=str, default="", help="extra unit shapes, e.g. 8192x1536,8192x8960")
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--no-coeffs", action="store_true")
+    a = ap.parse_args()
+    for fmt in a.fmts:
+        for lr in range(a.min_log2_rows, a.max_log2_rows + 1):
+            rows = 1 << lr
+            reps = a.reps if rows * a.cols * 2 < (1 << 30) else max(3, a.reps // 4)
+            print(json.dumps(codec_point(rows, a.cols, fmt, reps)), flush=True)
+            torch.cuda.empty_cache()
+    for shp in [s for s in a.shapes.split(",") if s]:
+        r, c = (int(v) for v in shp.split("x"))
+        for fmt in a.fmts:
+            print(json.dumps(codec_point(r, c, fmt, a.reps)), flush=True)
+            torch.cuda.empty_cache()
+    if not a.no_coeffs:
+        for ls in range(16, 25):
+            print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
+
+
+if __name__ == "__main__":
+    main()

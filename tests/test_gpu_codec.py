@@ -104,6 +104,11 @@ def test_special_values_inside_gaussian_data(fmt):
     x[8, 0] = 0x43E8                                   # 464: last value that still rounds to 448 unscaled
     x[9, 0] = 0x43E9                                   # 466: overflows to NaN unscaled
     x[10, 3] = 0xC3E9
+    # blocks whose absmax sits at / just above the point where Q / amax stops fitting fp32
+    for row, bits in ((11, 0x03E0), (12, 0x03E1), (13, 0x02FE), (14, 0x02FF), (15, 0x0380), (16, 0x0400)):
+        x[row, 384:448] = 0x0001
+        x[row, 400] = bits
+        x[row, 401] = bits | 0x8000
     check_roundtrip(x, fmt)
 
 

@@ -282,3 +282,21 @@ def test_leading_dimension_and_shape_errors():
         assert np.array_equal(out[:, :192], oracle.recover(c1, s1, fmt, blk)) and np.all(out[:, 192:] == 0)
     with pytest.raises(oracle.OracleError):
         oracle.compress(_acts(5, 2, 96), FMT_E4M3FN_BLK, 64)
+
+
+@pytest.mark.parametrize("fmt,Q,last_unit", [(FMT_E4M3FN_BLK, 448.0, 0x03E0), (FMT_INT8_BLK, 127.0, 0x02FE)])
+def test_blk_unit_scale_threshold(fmt, Q, last_unit):
+    """s = inv = 1 exactly when fl32(Q / amax) overflows: amax <= 1.75 * 2^-120 (Q = 448) resp.
+    1.984375 * 2^-122 (Q = 127); the next bf16 value already gets a finite reciprocal."""
+    for bits, unit in ((last_unit, True), (last_unit + 1, False), (1, True), (last_unit - 1, True)):
+        x = np.full((1, 64), 0x0001, np.uint16)
+        x[0, 7] = bits
+        amax = float(bits_to_f32(np.array([bits], np.uint16))[0])
+        with np.errstate(over="ignore"):
+            overflow = np.isinf(np.float32(Q) / np.float32(amax))
+        assert overflow == unit
+        c, s = oracle.compress(x, fmt, 64)
+        if unit:
+            assert s[0, 0] == 1.0 and np.all(c == 0)
+        else:
+            assert s[0, 0] == np.float32(amax) / np.float32(Q) and (c[0, 7] & 0x7F) == (0x7E if fmt == FMT_E4M3FN_BLK else 127)
