@@ -14,8 +14,9 @@
  *   - Returns an int status (HILORE_OK = 0).  Never throws, aborts or traps.
  *   - Every pointer is a DEVICE pointer owned by the caller, valid until the work enqueued
  *     by the call has finished, unless its comment says "host".
- *   - The library allocates nothing and keeps no state between calls (the one exception is
- *     stated at its declaration).  Work is enqueued on `stream` (a cudaStream_t passed as
+ *   - The library allocates nothing and keeps no data between calls (the one exception is stated at
+ *     its declaration); it only remembers immutable device properties (SM count, CTAs per SM of its
+ *     kernels) after the first call on a device.  Work is enqueued on `stream` (a cudaStream_t passed as
  *     void*; NULL = the legacy default stream) and the call returns without synchronising.
  *     HILORE_CUDA reports a launch error seen by cudaGetLastError, nothing asynchronous.
  *   - Tensors are row-major.  bf16 tensors are passed as void* (16-bit patterns).

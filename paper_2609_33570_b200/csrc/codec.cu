@@ -136,9 +136,7 @@ template <typename K> static int launch_one(K kernel, CodecWork wk, int64_t tota
 {
     wk.prefetch = prefetch;
     wk.split_global = env_int("HILORE_SPLIT_GLOBAL", 0);
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kCodecThreads, 0) != cudaSuccess || per_sm <= 0)
-        per_sm = 2;
+    int per_sm = ctas_per_sm(kernel, kCodecThreads, 0, 2);
     const int cap = env_int("HILORE_PER_SM", 0);
     if (cap > 0 && cap < per_sm)
         per_sm = cap;

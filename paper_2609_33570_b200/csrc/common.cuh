@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/hilore.h"
 
 #if defined(__CUDA_ARCH__) && (__CUDA_ARCH__ < 1000)
@@ -136,15 +138,65 @@ __device__ __forceinline__ float warp_sum(float v)
 
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// Number of SMs of the current device (queried each call; the library keeps no state).
+// Immutable properties of the devices, looked up once per device and process (no device memory involved).
+struct LaunchCache {
+    static constexpr int kMaxDevices = 64, kMaxKernels = 64;
+    std::mutex mu;
+    int sms[kMaxDevices] = {};
+    struct Entry {
+        const void *kernel;
+        int device, per_sm;
+    } occ[kMaxKernels] = {};
+    int n_occ = 0;
+};
+inline LaunchCache &launch_cache()
+{
+    static LaunchCache c;
+    return c;
+}
+
+inline int current_device()
+{
+    int dev = 0;
+    return cudaGetDevice(&dev) == cudaSuccess ? dev : 0;
+}
+
+// Number of SMs of the current device.
 inline int sm_count()
 {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess)
-        return 148;
+    const int dev = current_device();
+    LaunchCache &c = launch_cache();
+    if (dev >= 0 && dev < LaunchCache::kMaxDevices && c.sms[dev] > 0)
+        return c.sms[dev];
+    int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
         return 148;
+    if (dev >= 0 && dev < LaunchCache::kMaxDevices) {
+        std::lock_guard<std::mutex> lock(c.mu);
+        c.sms[dev] = sms;
+    }
     return sms;
+}
+
+// Resident CTAs per SM of `kernel` at `threads` threads and `smem` bytes of dynamic shared memory.
+template <typename K> inline int ctas_per_sm(K kernel, int threads, size_t smem, int fallback)
+{
+    const int dev = current_device();
+    LaunchCache &c = launch_cache();
+    const void *key = reinterpret_cast<const void *>(kernel);
+    {
+        std::lock_guard<std::mutex> lock(c.mu);
+        for (int i = 0; i < c.n_occ; ++i)
+            if (c.occ[i].kernel == key && c.occ[i].device == dev)
+                return c.occ[i].per_sm;
+    }
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess || per_sm <= 0)
+        return fallback;
+    std::lock_guard<std::mutex> lock(c.mu);
+    if (c.n_occ < LaunchCache::kMaxKernels)
+        c.occ[c.n_occ++] = {key, dev, per_sm};
+    return per_sm;
 }
 
 } // namespace hilore
