@@ -1,0 +1,207 @@
+"""Parity at the benchmark's full sizes and in its launch configuration, on sampled rows.
+
+A row's codes, scales, token RMS and reconstruction depend on that row only, so the oracle can check any
+sample of rows of units far too large to run through it whole.  Inputs are drawn on the device with the
+same recipe as the host generators (N(0,1), 1 % of the channels x20)."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+import oracle
+from paper_2609_33570_b200 import api, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+R, H, L = api.ACT_R, api.ACT_H, api.ACT_L
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def check_rows(x, codes, scales, out, rms, rows, fmt, what=("codes", "rms", "out")):
+    """Oracle check of the given row indices of one unit (device tensors)."""
+    idx = torch.as_tensor(sorted(set(int(r) for r in rows)), device=x.device)
+    xb = bits(x[idx])
+    blk = 0 if fmt == api.FMT_E4M3FN_RAW else 64
+    oc, osc = oracle.compress(xb, fmt, blk)
+    if "codes" in what:
+        assert np.array_equal(codes[idx].cpu().numpy(), oc)
+        if blk:
+            assert np.array_equal(scales[idx].cpu().numpy().view(np.uint32), osc.view(np.uint32))
+    if "rms" in what:
+        assert G.rel_err(rms[idx].cpu().numpy(), oracle.row_rms(xb)).max() <= 1e-5
+    if "out" in what:
+        assert np.array_equal(bits(out[idx]), oracle.recover(oc, osc, fmt, blk))
+
+
+def sample_rows(rng, rows, n=24):
+    return [0, 1, rows // 2, rows - 2, rows - 1] + rng.integers(0, rows, n).tolist()
+
+
+def test_bench_step_1p5B_shaped_microbatch():
+    """configs[1]: the exact object bench.py times (84 units, one launch per phase, all L)."""
+    dev = torch.device("cuda", 0)
+    wl = bench.Workload(api, synth, seed=0, device=dev)
+    for t in wl.codes + wl.out:
+        t.fill_(0xA5 if t.dtype == torch.uint8 else -1.0)
+    wl.step(3)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(0)
+    assert wl.action.cpu().tolist() == [L] * wl.U and wl.recompute.cpu().tolist() == [0] * wl.U
+    want_bytes = [r * c + 4 * r * c // 64 for r, c in wl.shapes]
+    assert wl.retained.cpu().tolist() == want_bytes
+    for u in (0, 1, 2, 41, 42, 43, 81, 82, 83):
+        check_rows(wl.x[u], wl.codes[u], wl.scales[u], wl.out[u], wl.rms[u], sample_rows(rng, wl.rows), api.FMT_E4M3FN_BLK)
+    # coefficients of microbatch 3 and the exposure of all 84 units (token RMS as the GPU wrote it)
+    ro = wl.ro
+    sl = slice(3 * bench.MB_RESP, 4 * bench.MB_RESP)
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, _, _ = oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=ro.n_valid)
+    got_w = wl.omega.cpu().numpy()
+    assert G.rel_err(got_w, w).max() <= 1e-5
+    oE, _ = oracle.unit_exposure(got_w, ro.mask[sl], wl.rms.cpu().numpy())
+    assert G.rel_err(wl.exposure.cpu().numpy(), oE).max() <= 1e-5
+    psi = (wl.kappa.cpu().numpy() * wl.exposure.cpu().numpy()).astype(np.float32) * wl.ebar.cpu().numpy()
+    assert np.array_equal(wl.psi.cpu().numpy().view(np.uint32), psi.view(np.uint32))
+    # every byte of every output was written: no canary left in a random sample of code rows
+    for u in (5, 50):
+        assert not bool((wl.scales[u] == 0).all())
+    del wl
+    torch.cuda.empty_cache()
+
+
+def test_7B_shaped_mixed_plan():
+    """configs[2]: 84 units [16384, 3584|3584|18944], candidate plan all H, thresholds at the 50 % / 70 %
+    quantiles of psi (42 L / 17 R / 25 H), post-forward encode and recovery of the L units only."""
+    dev = torch.device("cuda", 0)
+    rows, layers = 16384, 28
+    shapes = synth.layer_unit_shapes("7B", rows, layers)
+    U = len(shapes)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1)
+    x = [synth.activation_unit_device(gen, r, c, dev) for r, c in shapes]
+    codes = [torch.full((r, c), 0xA5, dtype=torch.uint8, device=dev) for r, c in shapes]
+    scales = [torch.full((r, c // 64), -7.0, dtype=torch.float32, device=dev) for r, c in shapes]
+    out = [torch.full((r, c), -3.0, dtype=torch.bfloat16, device=dev) if c < 10000 else None for r, c in shapes]
+    big_out = torch.full((rows, 18944), -3.0, dtype=torch.bfloat16, device=dev)   # shared by the wide units (memory)
+    rms = torch.full((U, rows), -1.0, dtype=torch.float32, device=dev)
+    units = [dict(x=x[i], codes=codes[i], scales=scales[i], out=out[i] if out[i] is not None else big_out,
+                  row_rms=rms[i], rows=r, cols=c, fmt=api.FMT_E4M3FN_BLK, block=64) for i, (r, c) in enumerate(shapes)]
+    udev, uhost = api.make_unit_table(units, dev)
+    avail = torch.full((U,), H, dtype=torch.uint8, device=dev)
+    action = torch.zeros(U, dtype=torch.uint8, device=dev)
+    rec = torch.zeros(U, dtype=torch.uint8, device=dev)
+    retained = torch.zeros(U, dtype=torch.int64, device=dev)
+    psi = torch.zeros(U, dtype=torch.float32, device=dev)
+    expo = torch.zeros(U, dtype=torch.float32, device=dev)
+    call = lambda phase, **k: api.hilore_plan_apply(udev, uhost, U, phase, k.get("E"), k.get("kappa"), k.get("ebar"),
+                                                    k.get("lo", 0.0), k.get("hi", 0.0), avail, action, k.get("psi"), rec,
+                                                    retained)
+    call(api.PHASE_CAPTURE)                                   # q = H everywhere: token RMS only
+    torch.cuda.synchronize()
+    assert all(bool((c[:2] == 0xA5).all()) for c in codes[:6])
+    # microbatch 5 of 256: 8 responses x 2048 slots; G = 16, so a prompt group spans two microbatches
+    ro = synth.rollout(2, 16, 16, 2048)
+    mb, n_mb = 5, 8
+    sl = slice(mb * n_mb, (mb + 1) * n_mb)
+    t = lambda a: torch.from_numpy(a).to(dev)
+    omega = torch.empty((n_mb, 2048), dtype=torch.float32, device=dev)
+    api.hilore_grpo_coeffs(t(ro.rewards), ro.n_resp, 16, mb * n_mb, n_mb, 2048, t(ro.logp_new[sl]), t(ro.logp_old[sl]), None,
+                           t(ro.mask[sl]), 2048 * 128 * 16, None, 0.2, 0.0, 1e-6, None, omega, None, None)
+    nws = api.hilore_workspace_bytes(U, rows)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+    api.hilore_unit_exposure(omega, t(ro.mask[sl]), n_mb, 2048, rms, U, rows, 0, 1e-8, expo, None, ws, nws)
+    kappa = torch.from_numpy(np.random.default_rng(3).uniform(0.5, 2.0, U).astype(np.float32)).to(dev)
+    ebar = torch.full((U,), 0.0266, dtype=torch.float32, device=dev)
+    E = expo.cpu().numpy()
+    oE, _ = oracle.unit_exposure(omega.cpu().numpy(), ro.mask[sl], rms.cpu().numpy())
+    assert G.rel_err(E, oE).max() <= 1e-5
+    psi_h = (kappa.cpu().numpy() * E).astype(np.float32) * ebar.cpu().numpy()
+    srt = np.sort(psi_h)
+    lo, hi = float((srt[41] + srt[42]) / 2), float((srt[U - 26] + srt[U - 25]) / 2)
+    call(api.PHASE_DECIDE, E=expo, kappa=kappa, ebar=ebar, lo=lo, hi=hi, psi=psi)
+    a = action.cpu().numpy()
+    oa, opsi, orec, oret = oracle.plan(E, kappa.cpu().numpy(), ebar.cpu().numpy(), lo, hi, [H] * U, [s[0] for s in shapes],
+                                       [s[1] for s in shapes], [1] * U, [64] * U)
+    assert np.array_equal(a, oa) and np.array_equal(psi.cpu().numpy().view(np.uint32), opsi.view(np.uint32))
+    assert np.array_equal(rec.cpu().numpy(), orec) and np.array_equal(retained.cpu().numpy().view(np.uint64), oret)
+    assert [(a == v).sum() for v in (L, H, R)] == [42, 25, 17]
+    call(api.PHASE_ENCODE)
+    call(api.PHASE_RECOVER)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(4)
+    narrow_L = [u for u in range(U) if a[u] == L and shapes[u][1] < 10000]
+    wide_L = [u for u in range(U) if a[u] == L and shapes[u][1] > 10000]
+    for u in narrow_L[:3] + narrow_L[-2:]:
+        check_rows(x[u], codes[u], scales[u], out[u], rms[u], sample_rows(rng, rows, 12), api.FMT_E4M3FN_BLK)
+    for u in wide_L[:2] + wide_L[-1:]:
+        check_rows(x[u], codes[u], scales[u], None, rms[u], sample_rows(rng, rows, 8), api.FMT_E4M3FN_BLK, what=("codes", "rms"))
+    if wide_L:   # the shared reconstruction buffer holds the last wide L unit
+        u = wide_L[-1]
+        check_rows(x[u], codes[u], scales[u], big_out, rms[u], sample_rows(rng, rows, 8), api.FMT_E4M3FN_BLK)
+    for u in [v for v in range(U) if a[v] != L][:8]:          # H keeps its bundle, R is recomputed: nothing written
+        assert bool((codes[u] == 0xA5).all()) and bool((scales[u] == -7.0).all())
+        if out[u] is not None:
+            assert bool((out[u] == -3.0).all())
+        check_rows(x[u], None, None, None, rms[u], sample_rows(rng, rows, 6), api.FMT_E4M3FN_BLK, what=("rms",))
+    del x, codes, scales, out, big_out
+    torch.cuda.empty_cache()
+
+
+def test_variable_length_rollout_batch_full_size():
+    """configs[3]: 256 prompts x G=8 x 4096 slots, lengths U{128..4096}, rewards U[0,1), 13 equal-reward groups."""
+    ro = synth.rollout(0, 256, 8, 4096, rewards="uniform", lengths="uniform", equal_group_fraction=0.05)
+    got = G.grpo_coeffs(ro, N_on_device=True, extras=False)
+    assert got["N"] == ro.n_valid
+    adv = oracle.group_advantages(ro.rewards, 8)
+    w, r, chi = oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, None, ro.mask, N_norm=ro.n_valid)
+    hi, lo = np.float32(1.2), np.float32(0.8)
+    near = (np.abs(r - hi) <= 4 * np.spacing(hi)) | (np.abs(r - lo) <= 4 * np.spacing(lo))
+    assert G.rel_err(got["omega"][~near], w[~near]).max() <= 1e-5
+    assert near.sum() < 50
+    Rg = ro.rewards.reshape(-1, 8)
+    eq = np.where(Rg.max(axis=1) == Rg.min(axis=1))[0]
+    assert len(eq) == 13
+    for g in eq:
+        assert np.all(got["omega"][g * 8:(g + 1) * 8] == 0)
+    assert np.all(got["omega"][ro.mask == 0] == 0)
+    # one microbatch of 4 responses: masked exposure over a [16384, 3584] unit's token RMS
+    rng = np.random.default_rng(1)
+    x = synth.activation_unit(rng, 16384, 3584)
+    _, _, rms = G.compress(x, api.FMT_E4M3FN_BLK)
+    om = np.ascontiguousarray(got["omega"][8:12])
+    E, sw = G.unit_exposure(om, np.ascontiguousarray(ro.mask[8:12]), rms[None, :])
+    oE, osw = oracle.unit_exposure(om, np.ascontiguousarray(ro.mask[8:12]), oracle.row_rms(x)[None, :])
+    assert G.rel_err(E, oE).max() <= 1e-5 and abs(sw - osw) <= 1e-5 * osw
+
+
+def test_4GiB_unit_uses_64_bit_offsets():
+    """configs[4], top end: one unit of 2^31 elements ([524288, 4096] bf16 = 4 GiB), both formats."""
+    dev = torch.device("cuda", 0)
+    rows, cols = 1 << 19, 4096
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(5)
+    base = synth.activation_unit_device(gen, 1 << 14, cols, dev)
+    x = base.repeat(rows // base.shape[0], 1)
+    x[-1, -64:] = 3.0            # make the very last block distinctive
+    x[rows // 2 + 1, :64] = -5.0
+    rng = np.random.default_rng(6)
+    sample = sample_rows(rng, rows, 16) + [rows // 2, rows // 2 + 1, (1 << 18) + 1]
+    for fmt in (api.FMT_E4M3FN_BLK, api.FMT_E4M3FN_RAW):
+        blk = 64 if fmt == api.FMT_E4M3FN_BLK else 0
+        codes = torch.full((rows, cols), 0xA5, dtype=torch.uint8, device=dev)
+        scales = torch.full((rows, cols // 64), -7.0, dtype=torch.float32, device=dev) if blk else None
+        rms = torch.full((rows,), -1.0, dtype=torch.float32, device=dev)
+        out = torch.full((rows, cols), -3.0, dtype=torch.bfloat16, device=dev)
+        api.hilore_compress(x, rows, cols, cols, fmt, blk, codes, scales, rms)
+        api.hilore_recover(codes, scales, rows, cols, fmt, blk, out, cols)
+        torch.cuda.synchronize()
+        check_rows(x, codes, scales, out, rms, sample, fmt)
+        assert not bool((rms < 0).any())                      # every row was visited
+        # xor-fold of the codes: the tiled repetition of `base` must give identical code tiles
+        first = codes[: base.shape[0]]
+        assert bool((codes[3 * base.shape[0]: 4 * base.shape[0]] == first).all())
+        del codes, scales, rms, out
+        torch.cuda.empty_cache()
