@@ -26,6 +26,7 @@ struct CodecWork {
     const uint8_t *avail;     // q_u
     const uint8_t *action;    // a_u
     int prefetch;             // iterations of L2 prefetch run-ahead (0 = none)
+    int64_t seg_bytes;        // size of the window all CTAs sweep together
 };
 
 __device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
@@ -48,22 +49,28 @@ __device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
 
 
 // ---- work split ----
-// Every CTA takes the same share of every unit the launch is gated into: rows [rows*c/nC, rows*(c+1)/nC).
-// All CTAs therefore sweep one unit together (measured faster on B200 than giving each CTA one large
-// private slice of the whole launch: 5.9 vs 5.3 TB/s for compress) and finish together.
+// A unit is swept in equal segments of about `seg_bytes` of bf16 (units up to 1.5 x that size in one piece);
+// every CTA takes the same share of every segment: rows [n*c/nC, n*(c+1)/nC) of its n rows.  All CTAs
+// therefore work inside one window of memory at a time and finish together -- measured faster on B200 than
+// giving each CTA one large private slice of a unit or of the whole launch.
 struct Job {
     hilore_unit u;
     int op;
-    int64_t r0, r1; // this CTA's rows of the unit
+    int64_t r0, r1; // this CTA's rows of the current segment
 };
 
-__device__ __forceinline__ bool next_job(const CodecWork &wk, int &ui, Job &j)
+struct JobCursor {
+    int ui = 0;          // next unit
+    int64_t seg_row = 0; // first row of the next segment of unit ui
+};
+
+__device__ __forceinline__ bool next_job(const CodecWork &wk, JobCursor &cur, Job &j)
 {
-    for (; ui < wk.U; ++ui) {
-        j.op = unit_op(wk, ui);
+    for (; cur.ui < wk.U; ++cur.ui, cur.seg_row = 0) {
+        j.op = unit_op(wk, cur.ui);
         if (j.op == OP_NONE)
             continue;
-        j.u = wk.units ? wk.units[ui] : wk.single;
+        j.u = wk.units ? wk.units[cur.ui] : wk.single;
         const hilore_unit &u = j.u;
         const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
         if ((j.op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (j.op == OP_STATS && (!u.x || !u.row_rms)) ||
@@ -71,12 +78,18 @@ __device__ __forceinline__ bool next_job(const CodecWork &wk, int &ui, Job &j)
             continue; // the unit lacks a buffer this operation needs: leave it untouched
         if (j.op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
             j.u.row_rms = nullptr; // token magnitudes were collected at capture time
-        j.r0 = (u.rows * (int64_t)blockIdx.x) / gridDim.x;
-        j.r1 = (u.rows * (int64_t)(blockIdx.x + 1)) / gridDim.x;
-        if (j.r0 >= j.r1)
-            continue;
-        ++ui;
-        return true;
+        // equal segments, as close to seg_bytes each as the unit's size allows
+        const int64_t unit_bytes = u.rows * u.cols * 2;
+        const int64_t nseg = max((int64_t)1, (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes);
+        const int64_t seg_rows = max((int64_t)gridDim.x, (u.rows + nseg - 1) / nseg);
+        while (cur.seg_row < u.rows) {
+            const int64_t s0 = cur.seg_row, n = min(seg_rows, u.rows - s0);
+            cur.seg_row += n;
+            j.r0 = s0 + (n * (int64_t)blockIdx.x) / gridDim.x;
+            j.r1 = s0 + (n * (int64_t)(blockIdx.x + 1)) / gridDim.x;
+            if (j.r0 < j.r1)
+                return true; // the cursor already points at the next segment
+        }
     }
     return false;
 }
