@@ -82,17 +82,18 @@ def main():
     ap.add_argument("--shapes", type=str, default="", help="extra unit shapes, e.g. 8192x1536,8192x8960")
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--no-coeffs", action="store_true")
+    ap.add_argument("--no-rms", action="store_true", help="compress without the fused token RMS")
     a = ap.parse_args()
     for fmt in a.fmts:
         for lr in range(a.min_log2_rows, a.max_log2_rows + 1):
             rows = 1 << lr
             reps = a.reps if rows * a.cols * 2 < (1 << 30) else max(3, a.reps // 4)
-            print(json.dumps(codec_point(rows, a.cols, fmt, reps)), flush=True)
+            print(json.dumps(codec_point(rows, a.cols, fmt, reps, with_rms=not a.no_rms)), flush=True)
             torch.cuda.empty_cache()
     for shp in [s for s in a.shapes.split(",") if s]:
         r, c = (int(v) for v in shp.split("x"))
         for fmt in a.fmts:
-            print(json.dumps(codec_point(r, c, fmt, a.reps)), flush=True)
+            print(json.dumps(codec_point(r, c, fmt, a.reps, with_rms=not a.no_rms)), flush=True)
             torch.cuda.empty_cache()
     if not a.no_coeffs:
         for ls in range(16, 25):
