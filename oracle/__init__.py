@@ -42,6 +42,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.orc_grpo_objective.restype = C.c_double
         _lib.orc_relative_error.restype = C.c_double
+        _lib.orc_risk_budget.restype = C.c_double
     return _lib
 
 
@@ -174,3 +175,23 @@ def plan(exposure, kappa, ebar, tau_lo, tau_hi, avail, rows, cols, fmt, block, a
                           _p(cols, np.int64), _p(fmt, np.int32), _p(block, np.int32), _p(action, np.uint8),
                           _p(psi, np.float32), _p(rec, np.uint8), _p(ret, np.uint64)))
     return action, psi, rec, ret
+
+
+def allocate(psi, dtau, dmem, avail, M_res, delta_b, N=1024):
+    """The paper's DP allocator.  dtau, dmem: [U, 3] by action code (R, H, L).  -> (action[U], totals[3])
+    with totals = (utility of the selection, its memory cost, its risk)."""
+    psi = np.ascontiguousarray(psi, np.float32)
+    U = psi.size
+    dtau = np.ascontiguousarray(dtau, np.float64).reshape(U, 3)
+    dmem = np.ascontiguousarray(dmem, np.float64).reshape(U, 3)
+    avail = np.ascontiguousarray(avail, np.uint8)
+    action = np.zeros(U, np.uint8)
+    totals = np.zeros(3, np.float64)
+    _check(lib().orc_allocate(C.c_int32(U), _p(psi, np.float32), _p(dtau, np.float64), _p(dmem, np.float64),
+                              _p(avail, np.uint8), C.c_double(M_res), C.c_double(delta_b), C.c_int32(N),
+                              _p(action, np.uint8), _p(totals, np.float64)))
+    return action, totals
+
+
+def risk_budget(delta, N_b, N_total) -> float:
+    return float(lib().orc_risk_budget(C.c_double(delta), C.c_int64(N_b), C.c_int64(N_total)))

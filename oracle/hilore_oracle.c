@@ -29,11 +29,16 @@
  *                         actions" (exhaustive), hand example.  The threshold
  *                         rule that picks the desired action is NOT in the paper
  *                         (its allocator is a knapsack DP): "parity unpinned".
+ *   orc_allocate          the paper's allocator (knapsack DP on the conservative grid): exhaustive
+ *                         enumeration of all 3^U assignments of the discretised problem, the
+ *                         feasibility guarantee of upward rounding, the tie rules and the
+ *                         boundary cases, on hand examples
  *
  * Build: gcc -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #define ORC_OK 0
@@ -471,4 +476,114 @@ int orc_plan(const float *exposure, const float *kappa, const float *ebar, int32
         }
     }
     return ORC_OK;
+}
+
+/* ---------------------------------------------- joint H/L/R allocation (two-constraint knapsack) */
+/* The paper's allocator (Appendix "Joint Allocation and Schedule Validation"): maximise sum_u dtau_u(a_u)
+ * subject to sum_u dmem_u(a_u) <= M_res, sum_u d_u(a_u) <= delta_b with d(H) = d(R) = 0, d(L) = psi_u, and
+ * a_u in A_u(q_u), solved exactly on a grid of N intervals per axis with costs rounded UP:
+ *   h_B = M_res / N, h_d = delta_b / N, b_u(a) = ceil(dmem_u(a) / h_B), r_u(a) = ceil(d_u(a) / h_d);
+ *   F_0(0,0) = 0, else -inf;  F_i(j,k) = max over available a with b <= j, r <= k of
+ *   F_{i-1}(j - b, k - r) + dtau_i(a), candidates tried in the order R, H, L (the first maximum wins);
+ *   terminal state: the largest F_U(j,k); ties go to the lower risk state k, then the lower memory state j.
+ * Boundary cases: M_res == 0 leaves one memory state (only actions without memory cost);
+ * delta_b == 0 disables L and leaves one risk state.  R always has utility 0 and costs 0.
+ * dtau, dmem: [U][3] indexed by the action code (R = 0, H = 1, L = 2); column R is ignored.
+ * A NaN or negative psi makes L unavailable for that unit; negative memory costs count as 0.
+ * Plain triple loop over (unit, j, k) with a full predecessor table: O(U * (N+1)^2) time and memory.
+ * Pinned by exhaustive enumeration of all 3^U assignments (tests/test_oracle_allocate.py).           */
+int orc_allocate(int32_t U, const float *psi, const double *dtau, const double *dmem, const uint8_t *avail,
+                 double M_res, double delta_b, int32_t N, uint8_t *action, double *totals)
+{
+    if (U < 0 || N <= 0 || !psi || !dtau || !dmem || !avail || !action)
+        return ORC_INVALID;
+    if (!(M_res >= 0.0) || !(delta_b >= 0.0))
+        return ORC_INVALID;
+    const int KB = (M_res > 0.0) ? N + 1 : 1, KD = (delta_b > 0.0) ? N + 1 : 1;
+    const double hB = M_res / (double)N, hD = delta_b / (double)N;
+    const size_t S = (size_t)KB * (size_t)KD;
+    int *bc = (int *)malloc(sizeof(int) * 3 * (size_t)(U > 0 ? U : 1));
+    int *rc = (int *)malloc(sizeof(int) * 3 * (size_t)(U > 0 ? U : 1));
+    double *F0 = (double *)malloc(sizeof(double) * S), *F1 = (double *)malloc(sizeof(double) * S);
+    uint8_t *pred = (uint8_t *)malloc(S * (size_t)(U > 0 ? U : 1));
+    if (!bc || !rc || !F0 || !F1 || !pred) {
+        free(bc); free(rc); free(F0); free(F1); free(pred);
+        return ORC_INVALID;
+    }
+    /* integer costs; -1 marks an action that cannot be taken */
+    for (int u = 0; u < U; ++u) {
+        if (avail[u] > ACT_L) {
+            free(bc); free(rc); free(F0); free(F1); free(pred);
+            return ORC_INVALID;
+        }
+        for (int a = 0; a < 3; ++a) {
+            int ok = (a == ACT_R) || (avail[u] == ACT_H) || (avail[u] == ACT_L && a == ACT_L);
+            double dm = (a == ACT_R) ? 0.0 : dmem[u * 3 + a];
+            double d = (a == ACT_L) ? (double)psi[u] : 0.0;
+            if (dm < 0.0) dm = 0.0;
+            if (a == ACT_L && (!(d >= 0.0) || delta_b == 0.0)) ok = 0;   /* NaN / negative risk; zero budget */
+            if (!(dm == dm)) ok = 0;
+            long b = 0, r = 0;
+            if (ok) {
+                if (M_res > 0.0) b = (long)ceil(dm / hB); else if (dm > 0.0) ok = 0;
+                if (delta_b > 0.0) r = (long)ceil(d / hD);
+                if (b > N || r > N || b < 0 || r < 0) ok = 0;
+            }
+            bc[u * 3 + a] = ok ? (int)b : -1;
+            rc[u * 3 + a] = ok ? (int)r : -1;
+        }
+    }
+    for (size_t s = 0; s < S; ++s) F0[s] = -INFINITY;
+    F0[0] = 0.0;
+    for (int u = 0; u < U; ++u) {
+        for (int j = 0; j < KB; ++j)
+            for (int k = 0; k < KD; ++k) {
+                double best = -INFINITY;
+                uint8_t arg = 255;
+                for (int a = 0; a < 3; ++a) {            /* order R, H, L: the first maximum wins */
+                    int b = bc[u * 3 + a], r = rc[u * 3 + a];
+                    if (b < 0 || b > j || r > k) continue;
+                    double prev = F0[(size_t)(j - b) * KD + (k - r)];
+                    if (prev == -INFINITY) continue;
+                    double v = prev + ((a == ACT_R) ? 0.0 : dtau[u * 3 + a]);
+                    if (arg == 255 || v > best) {
+                        best = v;
+                        arg = (uint8_t)a;
+                    }
+                }
+                F1[(size_t)j * KD + k] = best;
+                pred[(size_t)u * S + (size_t)j * KD + k] = arg;
+            }
+        double *t = F0; F0 = F1; F1 = t;
+    }
+    /* terminal state: largest utility; ties: lower risk, then lower memory */
+    int bj = 0, bk = 0;
+    double bestF = -INFINITY;
+    int have = 0;
+    for (int k = 0; k < KD; ++k)
+        for (int j = 0; j < KB; ++j) {
+            double v = F0[(size_t)j * KD + k];
+            if (v == -INFINITY) continue;
+            if (!have || v > bestF) { bestF = v; bj = j; bk = k; have = 1; }
+        }
+    double tot_m = 0.0, tot_r = 0.0;
+    int j = bj, k = bk;
+    for (int u = U - 1; u >= 0; --u) {
+        uint8_t a = pred[(size_t)u * S + (size_t)j * KD + k];
+        if (a > ACT_L) a = ACT_R;                        /* cannot happen: R is always available */
+        action[u] = a;
+        j -= bc[u * 3 + a];
+        k -= rc[u * 3 + a];
+        if (a != ACT_R) tot_m += (dmem[u * 3 + a] < 0.0 ? 0.0 : dmem[u * 3 + a]);
+        if (a == ACT_L) tot_r += (double)psi[u];
+    }
+    if (totals) { totals[0] = bestF; totals[1] = tot_m; totals[2] = tot_r; }
+    free(bc); free(rc); free(F0); free(F1); free(pred);
+    return ORC_OK;
+}
+
+/* Microbatch risk budget delta_b = delta * N_b / sum_b' N_b' (Appendix "Online Scheduling"). */
+double orc_risk_budget(double delta, int64_t N_b, int64_t N_total)
+{
+    return (N_total > 0) ? delta * (double)N_b / (double)N_total : 0.0;
 }
