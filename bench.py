@@ -394,6 +394,8 @@ def main():
                 "traffic": None if ratio is None else ratio * nbytes}
 
     sweep = coeff_sweep_point(api, synth, device)
+    from paper_2609_33570_b200 import sweep as sweep_mod
+    alloc = sweep_mod.allocate_point(wl.U, 5)      # the paper's DP allocator on its 1025 x 1025 grid (not part of the step)
     out = {
         "metric": METRIC, "value": world * wl.bytes_step / ms_step / 1e6, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
@@ -412,6 +414,7 @@ def main():
             "coeffs_microbatch": {"ms": kern_ms["coeffs"], "tokens_per_s": wl.rows / kern_ms["coeffs"] * 1e3},
             "exposure": {"ms": kern_ms["exposure"], "gbs": wl.bytes_exposure / kern_ms["exposure"] / 1e6},
             "coeffs_2p24": sweep,
+            "allocate_dp_u84_n1024": {"ms": alloc["us"] / 1e3, "state_updates_per_s": alloc["state_updates_per_s"]},
         },
         "coeff_tokens_per_s": sweep["tokens_per_s"],
         "e2e": e2e,

@@ -189,6 +189,35 @@ int hilore_compress(const void *x, int64_t rows, int64_t cols, int64_t ld, int32
 int hilore_recover(const uint8_t *codes, const float *scales, int64_t rows, int64_t cols, int32_t fmt,
                    int32_t block, void *out, int64_t ld_out, void *stream);
 
+/*
+ * Joint H / L / R allocation: the paper's allocator (Section "Joint H/L/R Allocation", Eq. "joint-allocation";
+ * Appendix "Joint Allocation and Schedule Validation", Eqs. "allocation-grid", "allocation-integer-costs",
+ * "allocation-dp").  Maximise sum_u dtau_u(a_u) subject to sum_u dmem_u(a_u) <= M_res,
+ * sum_u d_u(a_u) <= delta_b with d(H) = d(R) = 0 and d(L) = psi_u, and a_u in A_u(q_u), exactly on the
+ * conservative grid: h_B = M_res / N, h_d = delta_b / N, b_u(a) = ceil(dmem_u(a) / h_B),
+ * r_u(a) = ceil(d_u(a) / h_d) (costs rounded up, so every grid-feasible assignment is feasible);
+ * F_0(0,0) = 0, F_i(j,k) = max_a F_{i-1}(j - b, k - r) + dtau_i(a), candidates in the order R, H, L (first
+ * maximum wins); terminal ties favour the lower risk state, then the lower memory state.  M_res == 0 leaves
+ * one memory state (only actions without memory cost); delta_b == 0 disables L.  A NaN or negative psi_u makes
+ * L unavailable for unit u; negative memory costs count as 0; R always has utility 0 and costs 0.
+ * FP64 utilities as in the paper.  Layer i of the DP is one data-parallel pass over the (N+1)^2 states.
+ *
+ *   psi      [U] fp32 (device), e.g. written by hilore_plan_apply(PHASE_DECIDE).
+ *   dtau, dmem   [U, 3] fp64 (device), indexed by the action code (R, H, L); column R is ignored.
+ *   avail    [U] u8: the candidate plan q_u.        M_res, delta_b  host scalars, >= 0 (else INVALID_ARG).
+ *   n_intervals  N; the paper uses 1024.
+ *   action   [U] u8 out.   recompute  opt [U] u8 (1 iff R).   totals  opt [3] fp64: utility, memory, risk of the
+ *            selection (8-byte aligned).
+ *   workspace    hilore_allocate_workspace_bytes(U, N) bytes, 256-byte aligned (two value tables and the
+ *            predecessor table; 105 MB for U = 84, N = 1024).
+ * hilore_risk_budget: the microbatch budget delta_b = delta * N_b / sum_b' N_b' (host arithmetic).
+ */
+int hilore_allocate(int32_t U, const float *psi, const double *dtau, const double *dmem, const uint8_t *avail,
+                    double M_res, double delta_b, int32_t n_intervals, uint8_t *action, uint8_t *recompute,
+                    double *totals, void *workspace, size_t workspace_bytes, void *stream);
+size_t hilore_allocate_workspace_bytes(int32_t U, int32_t n_intervals);
+double hilore_risk_budget(double delta, int64_t N_b, int64_t N_total);
+
 /* One recovery unit of a microbatch: where its bf16 bundle lives and where its L representation goes.
  * A DEVICE array of these is passed to hilore_plan_apply.  Field rules as in hilore_compress /
  * hilore_recover; `out` may equal `x` only if the caller no longer needs the original. */

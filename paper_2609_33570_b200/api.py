@@ -23,7 +23,8 @@ BLOCK = 64
 
 EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "hilore_grpo_coeffs",
            "hilore_unit_exposure", "hilore_workspace_bytes", "hilore_compress", "hilore_recover",
-           "hilore_plan_apply", "hilore_unit_exposure_static", "hilore_static_scratch_bytes")
+           "hilore_plan_apply", "hilore_unit_exposure_static", "hilore_static_scratch_bytes",
+           "hilore_allocate", "hilore_allocate_workspace_bytes", "hilore_risk_budget")
 
 
 class HiloreUnit(C.Structure):
@@ -68,11 +69,17 @@ def lib() -> C.CDLL:
         _lib.hilore_unit_exposure_static.argtypes = [vp, vp, i64, i64, vp, i32, i64, i32, f32, vp, vp, vp]
         _lib.hilore_static_scratch_bytes.restype = C.c_size_t
         _lib.hilore_static_scratch_bytes.argtypes = []
+        _lib.hilore_allocate.argtypes = [i32, vp, vp, vp, vp, C.c_double, C.c_double, i32, vp, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_allocate_workspace_bytes.restype = C.c_size_t
+        _lib.hilore_allocate_workspace_bytes.argtypes = [i32, i32]
+        _lib.hilore_risk_budget.restype = C.c_double
+        _lib.hilore_risk_budget.argtypes = [C.c_double, i64, i64]
         _lib.hilore_compress.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
         _lib.hilore_recover.argtypes = [vp, vp, i64, i64, i32, i32, vp, i64, vp]
         _lib.hilore_plan_apply.argtypes = [vp, vp, i32, i32, vp, vp, vp, f32, f32, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
-            if name not in ("hilore_status_string", "hilore_workspace_bytes", "hilore_static_scratch_bytes"):
+            if name not in ("hilore_status_string", "hilore_workspace_bytes", "hilore_static_scratch_bytes",
+                            "hilore_allocate_workspace_bytes", "hilore_risk_budget"):
                 getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -126,6 +133,22 @@ def hilore_unit_exposure(omega, mask, n_rows, T, row_rms, U, rms_ld, row_shift, 
                                     eps_alpha, _ptr(exposure), _ptr(sum_abs_omega), _ptr(workspace),
                                     workspace_bytes, _stream(stream))
     return _check(st, "hilore_unit_exposure", check)
+
+
+def hilore_allocate_workspace_bytes(U, n_intervals=1024):
+    return int(lib().hilore_allocate_workspace_bytes(U, n_intervals))
+
+
+def hilore_risk_budget(delta, N_b, N_total):
+    return float(lib().hilore_risk_budget(delta, N_b, N_total))
+
+
+def hilore_allocate(U, psi, dtau, dmem, avail, M_res, delta_b, n_intervals, action, recompute, totals, workspace,
+                    workspace_bytes, stream=None, check=True):
+    st = lib().hilore_allocate(U, _ptr(psi), _ptr(dtau), _ptr(dmem), _ptr(avail), M_res, delta_b, n_intervals,
+                               _ptr(action), _ptr(recompute), _ptr(totals), _ptr(workspace), workspace_bytes,
+                               _stream(stream))
+    return _check(st, "hilore_allocate", check)
 
 
 def hilore_static_scratch_bytes():

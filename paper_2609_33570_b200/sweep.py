@@ -73,6 +73,29 @@ def coeffs_point(log2_slots, reps, G=16, T=1024):
             "gbs": 13 * slots / t / 1e6}
 
 
+def allocate_point(U, reps, N=1024):
+    """The DP allocator on the paper's grid: U units, synthetic utilities / memory costs / risks."""
+    import numpy as np
+    rng = np.random.default_rng(U)
+    psi = torch.from_numpy(rng.uniform(0, 0.004, U).astype(np.float32)).cuda()
+    dmem = np.zeros((U, 3))
+    dmem[:, 1] = rng.uniform(20, 600, U)
+    dmem[:, 2] = dmem[:, 1] * 0.53
+    dtau = np.zeros((U, 3))
+    dtau[:, 1] = rng.uniform(-0.5, 4.0, U)
+    dtau[:, 2] = dtau[:, 1] - rng.uniform(0.05, 0.8, U)
+    M_res, delta_b = float(dmem[:, 1].sum() * 0.35), float(psi.sum().item() * 0.3)
+    dt, dm = torch.from_numpy(dtau).cuda(), torch.from_numpy(dmem).cuda()
+    avail = torch.full((U,), api.ACT_H, dtype=torch.uint8, device="cuda")
+    action = torch.zeros(U, dtype=torch.uint8, device="cuda")
+    nws = api.hilore_allocate_workspace_bytes(U, N)
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    fn = lambda: api.hilore_allocate(U, psi, dt, dm, avail, M_res, delta_b, N, action, None, None, ws, nws)
+    t = _time([fn], reps)
+    return {"kernel": "allocate", "U": U, "N": N, "us": t * 1e3, "state_updates_per_s": U * (N + 1) ** 2 / t * 1e3,
+            "workspace_mib": nws / 2 ** 20}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--cols", type=int, default=4096)
@@ -98,6 +121,8 @@ def main():
     if not a.no_coeffs:
         for ls in range(16, 25):
             print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
+        for U in (36, 84):
+            print(json.dumps(allocate_point(U, max(3, a.reps // 4))), flush=True)
 
 
 if __name__ == "__main__":
