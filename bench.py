@@ -217,54 +217,65 @@ def coeff_sweep_point(api, synth, device, log2_slots=24, reps=10):
 
 # ---------------------------------------------------------------- CPU oracle legs
 SAMPLE_LAYERS = 4
+SAMPLE_TEXT = (f"layers 0-{SAMPLE_LAYERS - 1} of one microbatch ({3 * SAMPLE_LAYERS} of the 84 units: per layer [8192,1536]x2 + "
+               f"[8192,8960]), coefficients of 8192 slots, exposure U={3 * SAMPLE_LAYERS}")
+REFERENCE_BUDGET_S = 120.0     # the whole `--impl reference` run is sized to end within about this time
 
 
-def oracle_sample_step(synth_mod, seed=0, layers=SAMPLE_LAYERS):
-    """The oracle on a bounded sample of the workload: the first `layers` layers' units of one microbatch
-    (compress with token RMS, recover), the microbatch's coefficients, and the exposure of those units.
-    Returns (seconds, algorithmic bytes of the sample)."""
+def oracle_sample_step(synth_mod, seed=0, layers=SAMPLE_LAYERS, rows=MB_RESP * T):
+    """The oracle on a bounded sample of the workload: the first `rows` token rows of the first `layers`
+    layers' units of one microbatch (compress with token RMS, recover), the coefficients of those token
+    slots, and the exposure of those units.  Returns (seconds, algorithmic bytes of the sample)."""
     import oracle
     rng = np.random.default_rng(seed)
-    rows = MB_RESP * T
     shapes = synth_mod.layer_unit_shapes(MODEL, rows, layers)
     xs = [synth_mod.activation_unit(rng, r, c) for r, c in shapes]
-    ro = synth_mod.rollout(seed, 8, G_, T)          # a slice of the rollout batch is enough for the sample
+    n_rows = max(1, rows // T)                      # responses the sampled token rows belong to
+    t_len = min(T, rows)
+    ro = synth_mod.rollout(seed, 8, G_, t_len)      # a slice of the rollout batch is enough for the sample
     oracle.lib()
     t0 = time.perf_counter()
     rms = []
-    recs = 0
     for x in xs:
         codes, scales = oracle.compress(x, oracle.FMT_E4M3FN_BLK, 64)
         rms.append(oracle.row_rms(x))
-        recs += oracle.recover(codes, scales, oracle.FMT_E4M3FN_BLK, 64).size
+        oracle.recover(codes, scales, oracle.FMT_E4M3FN_BLK, 64)
     adv = oracle.group_advantages(ro.rewards, G_)
-    omega, _, _ = oracle.grpo_coeffs(adv[:MB_RESP], ro.logp_new[:MB_RESP], ro.logp_old[:MB_RESP], None,
-                                     ro.mask[:MB_RESP], N_norm=P * G_ * T)
-    E, _ = oracle.unit_exposure(omega, ro.mask[:MB_RESP], np.stack(rms))
+    omega, _, _ = oracle.grpo_coeffs(adv[:n_rows], ro.logp_new[:n_rows], ro.logp_old[:n_rows], None,
+                                     ro.mask[:n_rows], N_norm=P * G_ * T)
+    E, _ = oracle.unit_exposure(omega, np.ascontiguousarray(ro.mask[:n_rows]), np.ascontiguousarray(np.stack(rms)[:, :n_rows * t_len]))
     dt = time.perf_counter() - t0
     nbytes = sum(codec_bytes(r, c, True, True) + codec_bytes(r, c, True, False) for r, c in shapes) \
-        + coeff_bytes(rows) + exposure_bytes(rows, len(shapes))
+        + coeff_bytes(n_rows * t_len) + exposure_bytes(n_rows * t_len, len(shapes))
     return dt, nbytes
 
 
-SAMPLE_TEXT = (f"layers 0-{SAMPLE_LAYERS - 1} of one microbatch ({3 * SAMPLE_LAYERS} of the 84 units: per layer [8192,1536]x2 + "
-               f"[8192,8960]), coefficients of 8192 slots, exposure U={3 * SAMPLE_LAYERS}")
-
-
 def run_reference(args):
+    """The tier's reference arm: the CPU oracle, as it stands, on the host cores.  Each step is a bounded
+    sample of the workload (the first rows of layer 0's three units + their coefficients and exposure),
+    sized from a short calibration so that warm-up + timed steps end within about two minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2609_33570_b200 import synth
+    cal_rows = 1024
+    oracle_sample_step(synth, seed=12344, layers=1, rows=64)          # loads the library, touches the allocator
+    w0 = time.perf_counter()
+    oracle_sample_step(synth, seed=12345, layers=1, rows=cal_rows)
+    rows_per_s = cal_rows / max(time.perf_counter() - w0, 1e-6)        # wall clock: input generation included
+    budget = REFERENCE_BUDGET_S / max(1, args.steps + args.warmup)
+    rows = int(min(MB_RESP * T, max(64, rows_per_s * budget * 0.8)))
+    rows -= rows % 64
     times = []
     nbytes = 0
     for i in range(args.warmup + args.steps):
-        dt, nbytes = oracle_sample_step(synth, seed=i)
+        dt, nbytes = oracle_sample_step(synth, seed=i, layers=1, rows=rows)
         if i >= args.warmup:
             times.append(dt)
     sec = sum(times) / len(times)
     val = nbytes / sec / 1e9
-    sample = SAMPLE_TEXT
+    sample = (f"first {rows} of 8192 token rows of layer 0's units ([.,1536]x2 + [.,8960]) of one microbatch, the "
+              f"coefficients of those {rows} slots, exposure U=3")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
