@@ -218,6 +218,23 @@ int hilore_allocate(int32_t U, const float *psi, const double *dtau, const doubl
 size_t hilore_allocate_workspace_bytes(int32_t U, int32_t n_intervals);
 double hilore_risk_budget(double delta, int64_t N_b, int64_t N_total);
 
+/*
+ * Calibration of the L action (initialisation time, on the calibration microbatches).
+ *   hilore_relative_error: e^L = ||x_hat - x||_2 / (||x||_2 + 1e-8) of one unit, operands widened to fp32 before
+ *   the subtraction and the norms (Eq. "calibration-metrics"); fp32 per 16 elements, fp64 across them, per-CTA
+ *   partial sums in fixed workspace slots, added in a fixed order (deterministic).
+ *     x, xhat  [rows, ld] / [rows, ld_hat] bf16, 32-byte aligned, ld % 16 == 0; cols % 16 == 0.
+ *     e_out    one fp64 on the device.    norms2   opt [2] fp64 on the device: ||x_hat - x||^2, ||x||^2.
+ *     workspace  hilore_relative_error_workspace_bytes() bytes, 16-byte aligned.
+ *   The mean reconstruction error ebar_u^L is the plain average of e^L over the calibration microbatches.
+ *   hilore_fit_kappa: kappa_c = argmin_{kappa >= 0} sum_i (y_i - kappa x_i)^2 = max(0, sum x y / sum x^2)
+ *   (Eq. "susceptibility"), x_i = E_{u,b} e^L_{u,b}; HOST arrays, host arithmetic; 0 if every x_i is 0.
+ */
+int hilore_relative_error(const void *x, const void *xhat, int64_t rows, int64_t cols, int64_t ld, int64_t ld_hat,
+                          double *e_out, double *norms2, void *workspace, size_t workspace_bytes, void *stream);
+size_t hilore_relative_error_workspace_bytes(void);
+double hilore_fit_kappa(const double *x, const double *y, int64_t n);
+
 /* One recovery unit of a microbatch: where its bf16 bundle lives and where its L representation goes.
  * A DEVICE array of these is passed to hilore_plan_apply.  Field rules as in hilore_compress /
  * hilore_recover; `out` may equal `x` only if the caller no longer needs the original. */

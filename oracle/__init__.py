@@ -43,6 +43,7 @@ def lib():
         _lib.orc_grpo_objective.restype = C.c_double
         _lib.orc_relative_error.restype = C.c_double
         _lib.orc_risk_budget.restype = C.c_double
+        _lib.orc_fit_kappa.restype = C.c_double
     return _lib
 
 
@@ -195,3 +196,9 @@ def allocate(psi, dtau, dmem, avail, M_res, delta_b, N=1024):
 
 def risk_budget(delta, N_b, N_total) -> float:
     return float(lib().orc_risk_budget(C.c_double(delta), C.c_int64(N_b), C.c_int64(N_total)))
+
+
+def fit_kappa(x, y) -> float:
+    x = np.ascontiguousarray(x, np.float64)
+    y = np.ascontiguousarray(y, np.float64)
+    return float(lib().orc_fit_kappa(_p(x, np.float64), _p(y, np.float64), C.c_int64(x.size)))

@@ -29,6 +29,9 @@
  *                         actions" (exhaustive), hand example.  The threshold
  *                         rule that picks the desired action is NOT in the paper
  *                         (its allocator is a knapsack DP): "parity unpinned".
+ *   orc_relative_error,
+ *   orc_fit_kappa         e^L against NumPy fp64 norms and its expected size on Gaussian data; kappa
+ *                         against a brute-force minimisation over a grid and exact lines
  *   orc_allocate          the paper's allocator (knapsack DP on the conservative grid): exhaustive
  *                         enumeration of all 3^U assignments of the discretised problem, the
  *                         feasibility guarantee of upward rounding, the tie rules and the
@@ -586,4 +589,19 @@ int orc_allocate(int32_t U, const float *psi, const double *dtau, const double *
 double orc_risk_budget(double delta, int64_t N_b, int64_t N_total)
 {
     return (N_total > 0) ? delta * (double)N_b / (double)N_total : 0.0;
+}
+
+/* Susceptibility fit kappa_c = argmin_{kappa >= 0} sum (y - kappa x)^2 (Eq. "susceptibility"): the closed
+ * form max(0, sum x y / sum x^2); 0 when every x is 0. */
+double orc_fit_kappa(const double *x, const double *y, int64_t n)
+{
+    double sxy = 0.0, sxx = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        sxy += x[i] * y[i];
+        sxx += x[i] * x[i];
+    }
+    if (!(sxx > 0.0))
+        return 0.0;
+    double k = sxy / sxx;
+    return k > 0.0 ? k : 0.0;
 }

@@ -24,7 +24,8 @@ BLOCK = 64
 EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "hilore_grpo_coeffs",
            "hilore_unit_exposure", "hilore_workspace_bytes", "hilore_compress", "hilore_recover",
            "hilore_plan_apply", "hilore_unit_exposure_static", "hilore_static_scratch_bytes",
-           "hilore_allocate", "hilore_allocate_workspace_bytes", "hilore_risk_budget")
+           "hilore_allocate", "hilore_allocate_workspace_bytes", "hilore_risk_budget",
+           "hilore_relative_error", "hilore_relative_error_workspace_bytes", "hilore_fit_kappa")
 
 
 class HiloreUnit(C.Structure):
@@ -74,12 +75,18 @@ def lib() -> C.CDLL:
         _lib.hilore_allocate_workspace_bytes.argtypes = [i32, i32]
         _lib.hilore_risk_budget.restype = C.c_double
         _lib.hilore_risk_budget.argtypes = [C.c_double, i64, i64]
+        _lib.hilore_relative_error.argtypes = [vp, vp, i64, i64, i64, i64, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_relative_error_workspace_bytes.restype = C.c_size_t
+        _lib.hilore_relative_error_workspace_bytes.argtypes = []
+        _lib.hilore_fit_kappa.restype = C.c_double
+        _lib.hilore_fit_kappa.argtypes = [vp, vp, i64]
         _lib.hilore_compress.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
         _lib.hilore_recover.argtypes = [vp, vp, i64, i64, i32, i32, vp, i64, vp]
         _lib.hilore_plan_apply.argtypes = [vp, vp, i32, i32, vp, vp, vp, f32, f32, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("hilore_status_string", "hilore_workspace_bytes", "hilore_static_scratch_bytes",
-                            "hilore_allocate_workspace_bytes", "hilore_risk_budget"):
+                            "hilore_allocate_workspace_bytes", "hilore_risk_budget",
+                            "hilore_relative_error_workspace_bytes", "hilore_fit_kappa"):
                 getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -149,6 +156,25 @@ def hilore_allocate(U, psi, dtau, dmem, avail, M_res, delta_b, n_intervals, acti
                                _ptr(action), _ptr(recompute), _ptr(totals), _ptr(workspace), workspace_bytes,
                                _stream(stream))
     return _check(st, "hilore_allocate", check)
+
+
+def hilore_relative_error_workspace_bytes():
+    return int(lib().hilore_relative_error_workspace_bytes())
+
+
+def hilore_relative_error(x, xhat, rows, cols, ld, ld_hat, e_out, norms2, workspace, workspace_bytes, stream=None,
+                          check=True):
+    st = lib().hilore_relative_error(_ptr(x), _ptr(xhat), rows, cols, ld, ld_hat, _ptr(e_out), _ptr(norms2),
+                                     _ptr(workspace), workspace_bytes, _stream(stream))
+    return _check(st, "hilore_relative_error", check)
+
+
+def hilore_fit_kappa(x, y):
+    """x, y: sequences of host floats (calibration pairs)."""
+    n = len(x)
+    ax = (C.c_double * n)(*[float(v) for v in x])
+    ay = (C.c_double * n)(*[float(v) for v in y])
+    return float(lib().hilore_fit_kappa(C.cast(ax, C.c_void_p), C.cast(ay, C.c_void_p), n))
 
 
 def hilore_static_scratch_bytes():

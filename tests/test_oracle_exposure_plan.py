@@ -135,3 +135,17 @@ def test_plan_threshold_example():
     E[3] = np.nan
     a, *_ = oracle.plan(E, kappa, ebar, 0.045, 0.075, avail, [8] * 10, [64] * 10, [1] * 10, [64] * 10)
     assert a[3] == ACT_R
+
+
+def test_fit_kappa_closed_form_against_grid_search():
+    """kappa = argmin_{kappa >= 0} sum (y - kappa x)^2 (Eq. "susceptibility")."""
+    rng = np.random.default_rng(0)
+    x = rng.uniform(0, 1, 50)
+    assert oracle.fit_kappa(x, 2.5 * x) == pytest.approx(2.5, rel=1e-12)      # exact line
+    assert oracle.fit_kappa(x, -3 * x) == 0.0                                 # constrained at zero
+    assert oracle.fit_kappa(np.zeros(4), np.ones(4)) == 0.0                   # no signal
+    y = 1.7 * x + rng.normal(0, 0.1, 50)
+    k = oracle.fit_kappa(x, y)
+    grid = np.linspace(0, 4, 40001)
+    loss = ((y[None, :] - grid[:, None] * x[None, :]) ** 2).sum(axis=1)
+    assert k == pytest.approx(grid[loss.argmin()], abs=2e-4)
