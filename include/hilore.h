@@ -111,6 +111,38 @@ int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, in
                        float *omega, float *ratio, uint8_t *clip_mask, void *stream);
 
 /*
+ * Score variants of the component ablations (paragraph "Component ablations"): hilore_grpo_coeffs with one
+ * more argument.  variant 0: omega as above.  variant 1 ("removing ratio/clipping"): chi_t r_t replaced by 1 in
+ * the policy contribution, omega_t = -(m_t / N) A + beta (m_t / N)(1 - exp(s_ref - s)).  variant 2: the
+ * advantage-only signal omega_t := m_t A, whose exposure is sum_t |A_t| alpha_t.  "Removing KL" is beta = 0;
+ * "removing activation weighting" is the sum_abs_omega output of hilore_unit_exposure; "removing
+ * susceptibility" is kappa = 1.  ratio and clip_mask are reported as in hilore_grpo_coeffs.
+ */
+int hilore_grpo_coeffs_variant(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                               int64_t n_rows, int64_t T, const float *logp_new, const float *logp_old,
+                               const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                               const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps, int32_t variant,
+                               float *adv_out, float *omega, float *ratio, uint8_t *clip_mask, void *stream);
+
+/*
+ * Structural sparsity of one record of coefficients (paragraph "Structural sparsity in diagnostic replays",
+ * Eq. "diagnostic-clipping").  Over the n = n_rows * T padded response slots:
+ *   counts[0] padding slots (m = 0);  counts[1] valid slots with zero advantage;  counts[2] valid slots with
+ *   nonzero advantage on a flat clipped branch, (A > 0 and r > 1 + eps) or (A < 0 and r < 1 - eps);
+ *   counts[3] slots whose coefficient is zero (padding counts as zero);  counts[4] = n, the common denominator.
+ *   top_share = share of sum |omega| carried by the ceil(0.1 n) slots of largest |omega| (exact: the k-th largest
+ *   value is found by a radix select on the bit patterns; ties at the threshold contribute as many copies as the
+ *   decile still needs).   sum_abs = sum |omega| over valid slots.
+ *   adv [n_rows], ratio / omega [n_rows, T] fp32, mask [n_rows, T] u8 (device); counts [5] int64, top_share,
+ *   sum_abs (opt) fp64 on the device, 8-byte aligned; workspace hilore_omega_diagnostics_workspace_bytes() bytes.
+ * Integer histograms and fixed-slot fp64 partial sums: the result is deterministic.
+ */
+int hilore_omega_diagnostics(const float *adv, const float *ratio, const uint8_t *mask, const float *omega,
+                             int64_t n_rows, int64_t T, float clip_eps, int64_t *counts, double *top_share,
+                             double *sum_abs, void *workspace, size_t workspace_bytes, void *stream);
+size_t hilore_omega_diagnostics_workspace_bytes(void);
+
+/*
  * Operational update exposure of U units over one microbatch
  * (Eq. "activation-token-weights", Eq. "mlp-weighted-exposure"):
  *     T_b = slots with mask = 1;  abar_u = mean_{t in T_b} a_{t,u}

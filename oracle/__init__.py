@@ -202,3 +202,29 @@ def fit_kappa(x, y) -> float:
     x = np.ascontiguousarray(x, np.float64)
     y = np.ascontiguousarray(y, np.float64)
     return float(lib().orc_fit_kappa(_p(x, np.float64), _p(y, np.float64), C.c_int64(x.size)))
+
+
+def grpo_coeffs_variant(adv_rows, logp_new, logp_old, logp_ref, mask, N_norm=0, clip_eps=0.2, beta=0.0, variant=0):
+    n_rows, T = logp_new.shape
+    adv_rows = np.ascontiguousarray(adv_rows, dtype=np.float32)
+    omega = np.empty((n_rows, T), np.float32)
+    ratio = np.empty((n_rows, T), np.float32)
+    chi = np.empty((n_rows, T), np.uint8)
+    _check(lib().orc_grpo_coeffs_variant(_p(adv_rows, np.float32), _p(logp_new, np.float32), _p(logp_old, np.float32),
+                                         _p(logp_ref, np.float32), _p(mask, np.uint8), C.c_int64(n_rows), C.c_int64(T),
+                                         C.c_int64(N_norm), C.c_float(clip_eps), C.c_float(beta), C.c_int32(variant),
+                                         _p(omega, np.float32), _p(ratio, np.float32), _p(chi, np.uint8)))
+    return omega, ratio, chi
+
+
+def omega_diagnostics(adv_rows, ratio, mask, omega, clip_eps=0.2):
+    """-> (counts[5] = padding, zero-advantage, clipped, zero-omega, slots; top-decile share; sum |omega|)."""
+    n_rows, T = omega.shape
+    adv_rows = np.ascontiguousarray(adv_rows, dtype=np.float32)
+    counts = np.zeros(5, np.int64)
+    share = C.c_double(0.0)
+    total = C.c_double(0.0)
+    _check(lib().orc_omega_diagnostics(_p(adv_rows, np.float32), _p(ratio, np.float32), _p(mask, np.uint8),
+                                       _p(omega, np.float32), C.c_int64(n_rows), C.c_int64(T), C.c_float(clip_eps),
+                                       _p(counts, np.int64), C.byref(share), C.byref(total)))
+    return counts, float(share.value), float(total.value)

@@ -32,6 +32,9 @@
  *   orc_relative_error,
  *   orc_fit_kappa         e^L against NumPy fp64 norms and its expected size on Gaussian data; kappa
  *                         against a brute-force minimisation over a grid and exact lines
+ *   orc_grpo_coeffs_variant, orc_omega_diagnostics   hand-worked record, identities of Remark 1 (beta = 0:
+ *                         zero-omega slots = padding + zero-advantage + clipped), NumPy sort for the
+ *                         top-decile share, closed forms for uniform / one-hot |omega|
  *   orc_allocate          the paper's allocator (knapsack DP on the conservative grid): exhaustive
  *                         enumeration of all 3^U assignments of the discretised problem, the
  *                         feasibility guarantee of upward rounding, the tie rules and the
@@ -604,4 +607,84 @@ double orc_fit_kappa(const double *x, const double *y, int64_t n)
         return 0.0;
     double k = sxy / sxx;
     return k > 0.0 ? k : 0.0;
+}
+
+/* ------------------------------------------------ diagnostics and score variants on omega */
+/* Score variants of the component ablations: bit 0 replaces chi_t r_t by 1 in the policy contribution
+ * ("removing ratio/clipping"); bit 1 writes the advantage-only signal m_t A instead of omega (the summand of
+ * the advantage-only exposure sum_t |A_t| alpha_t).  "Removing KL" is beta = 0.  Ratio and clip indicator are
+ * reported as in orc_grpo_coeffs. */
+int orc_grpo_coeffs_variant(const float *adv, const float *logp_new, const float *logp_old, const float *logp_ref,
+                            const uint8_t *mask, int64_t n_rows, int64_t T, int64_t N_norm, float clip_eps, float beta,
+                            int32_t variant, float *omega, float *ratio, uint8_t *clip_mask)
+{
+    int st = orc_grpo_coeffs(adv, logp_new, logp_old, logp_ref, mask, n_rows, T, N_norm, clip_eps, beta, omega, ratio,
+                             clip_mask);
+    if (st != ORC_OK || variant == 0)
+        return st;
+    int64_t N = N_norm;
+    if (N <= 0) {
+        N = 0;
+        for (int64_t i = 0; i < n_rows * T; ++i) N += mask[i] ? 1 : 0;
+    }
+    for (int64_t i = 0; i < n_rows; ++i)
+        for (int64_t t = 0; t < T; ++t) {
+            int64_t k = i * T + t;
+            double m = mask[k] ? 1.0 : 0.0;
+            if (variant & 2) {
+                omega[k] = (float)(m * (double)adv[i]);
+                continue;
+            }
+            double w = -(m / (double)N) * (double)adv[i];               /* chi r -> 1 */
+            if (beta != 0.0f)
+                w += (double)beta * (m / (double)N) * (1.0 - exp((double)logp_ref[k] - (double)logp_new[k]));
+            omega[k] = (float)w;
+        }
+    return ORC_OK;
+}
+
+static int cmp_desc_float(const void *a, const void *b)
+{
+    float x = *(const float *)a, y = *(const float *)b;
+    return (x < y) - (x > y);
+}
+
+/* Structural sparsity of one record (diagnostic paragraph "Structural sparsity", Eq. "diagnostic-clipping"):
+ * counts[0] = padding slots (m = 0); counts[1] = valid slots with zero advantage; counts[2] = valid slots with
+ * nonzero advantage on a flat clipped branch, (A > 0 and r > 1 + eps) or (A < 0 and r < 1 - eps); counts[3] =
+ * slots with omega == 0; counts[4] = all padded response slots (the common denominator).  top_share = share of
+ * sum |omega| carried by the ceil(0.1 n) slots of largest |omega| (padding counts with zero coefficient). */
+int orc_omega_diagnostics(const float *adv, const float *ratio, const uint8_t *mask, const float *omega, int64_t n_rows,
+                          int64_t T, float clip_eps, int64_t *counts, double *top_share, double *sum_abs)
+{
+    if (!adv || !ratio || !mask || !omega || !counts || n_rows < 0 || T < 0)
+        return ORC_INVALID;
+    const int64_t n = n_rows * T;
+    const float hi = 1.0f + clip_eps, lo = 1.0f - clip_eps;
+    for (int c = 0; c < 5; ++c) counts[c] = 0;
+    counts[4] = n;
+    float *absw = (float *)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
+    if (!absw)
+        return ORC_INVALID;
+    double total = 0.0;
+    for (int64_t i = 0; i < n_rows; ++i)
+        for (int64_t t = 0; t < T; ++t) {
+            int64_t k = i * T + t;
+            float A = adv[i], r = ratio[k];
+            if (!mask[k]) counts[0]++;
+            else if (A == 0.0f) counts[1]++;
+            else if ((A > 0.0f && r > hi) || (A < 0.0f && r < lo)) counts[2]++;
+            float w = mask[k] ? fabsf(omega[k]) : 0.0f;
+            if (w == 0.0f) counts[3]++;
+            absw[k] = w;
+            total += (double)w;
+        }
+    qsort(absw, (size_t)n, sizeof(float), cmp_desc_float);
+    int64_t kk = (n * 1 + 9) / 10;                     /* ceil(0.1 n) */
+    double top = 0.0;
+    for (int64_t i = 0; i < kk; ++i) top += (double)absw[i];
+    free(absw);
+    if (top_share) *top_share = total > 0.0 ? top / total : 0.0;
+    if (sum_abs) *sum_abs = total;
+    return ORC_OK;
 }

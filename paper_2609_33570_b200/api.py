@@ -25,7 +25,8 @@ EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "h
            "hilore_unit_exposure", "hilore_workspace_bytes", "hilore_compress", "hilore_recover",
            "hilore_plan_apply", "hilore_unit_exposure_static", "hilore_static_scratch_bytes",
            "hilore_allocate", "hilore_allocate_workspace_bytes", "hilore_risk_budget",
-           "hilore_relative_error", "hilore_relative_error_workspace_bytes", "hilore_fit_kappa")
+           "hilore_relative_error", "hilore_relative_error_workspace_bytes", "hilore_fit_kappa",
+           "hilore_grpo_coeffs_variant", "hilore_omega_diagnostics", "hilore_omega_diagnostics_workspace_bytes")
 
 
 class HiloreUnit(C.Structure):
@@ -80,13 +81,19 @@ def lib() -> C.CDLL:
         _lib.hilore_relative_error_workspace_bytes.argtypes = []
         _lib.hilore_fit_kappa.restype = C.c_double
         _lib.hilore_fit_kappa.argtypes = [vp, vp, i64]
+        _lib.hilore_grpo_coeffs_variant.argtypes = [vp, i64, i32, i64, i64, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32, i32,
+                                                    vp, vp, vp, vp, vp]
+        _lib.hilore_omega_diagnostics.argtypes = [vp, vp, vp, vp, i64, i64, f32, vp, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_omega_diagnostics_workspace_bytes.restype = C.c_size_t
+        _lib.hilore_omega_diagnostics_workspace_bytes.argtypes = []
         _lib.hilore_compress.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, vp]
         _lib.hilore_recover.argtypes = [vp, vp, i64, i64, i32, i32, vp, i64, vp]
         _lib.hilore_plan_apply.argtypes = [vp, vp, i32, i32, vp, vp, vp, f32, f32, vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
             if name not in ("hilore_status_string", "hilore_workspace_bytes", "hilore_static_scratch_bytes",
                             "hilore_allocate_workspace_bytes", "hilore_risk_budget",
-                            "hilore_relative_error_workspace_bytes", "hilore_fit_kappa"):
+                            "hilore_relative_error_workspace_bytes", "hilore_fit_kappa",
+                            "hilore_omega_diagnostics_workspace_bytes"):
                 getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -128,6 +135,28 @@ def hilore_grpo_coeffs(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_ne
                                   clip_eps, beta, adv_eps, _ptr(adv_out), _ptr(omega), _ptr(ratio),
                                   _ptr(clip_mask), _stream(stream))
     return _check(st, "hilore_grpo_coeffs", check)
+
+
+def hilore_grpo_coeffs_variant(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask,
+                               N_norm, N_norm_dev, clip_eps, beta, adv_eps, variant, adv_out, omega, ratio, clip_mask,
+                               stream=None, check=True):
+    st = lib().hilore_grpo_coeffs_variant(_ptr(rewards), n_resp_total, G, resp_offset, n_rows, T, _ptr(logp_new),
+                                          _ptr(logp_old), _ptr(logp_ref), _ptr(mask), N_norm, _ptr(N_norm_dev),
+                                          clip_eps, beta, adv_eps, variant, _ptr(adv_out), _ptr(omega), _ptr(ratio),
+                                          _ptr(clip_mask), _stream(stream))
+    return _check(st, "hilore_grpo_coeffs_variant", check)
+
+
+def hilore_omega_diagnostics_workspace_bytes():
+    return int(lib().hilore_omega_diagnostics_workspace_bytes())
+
+
+def hilore_omega_diagnostics(adv, ratio, mask, omega, n_rows, T, clip_eps, counts, top_share, sum_abs, workspace,
+                             workspace_bytes, stream=None, check=True):
+    st = lib().hilore_omega_diagnostics(_ptr(adv), _ptr(ratio), _ptr(mask), _ptr(omega), n_rows, T, clip_eps,
+                                        _ptr(counts), _ptr(top_share), _ptr(sum_abs), _ptr(workspace), workspace_bytes,
+                                        _stream(stream))
+    return _check(st, "hilore_omega_diagnostics", check)
 
 
 def hilore_workspace_bytes(U, n_tok):

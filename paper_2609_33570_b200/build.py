@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhilore_b200.so")
-SOURCES = ["codec.cu", "grpo.cu", "allocate.cu", "calib.cu"]
+SOURCES = ["codec.cu", "grpo.cu", "allocate.cu", "calib.cu", "diag.cu"]
 HEADERS = ["common.cuh", "codec.cuh", os.path.join("..", "..", "include", "hilore.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]

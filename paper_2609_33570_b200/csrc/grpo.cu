@@ -89,7 +89,9 @@ __device__ float group_advantage(const float *rewards, int64_t resp, int G, floa
     return (float)(((double)__ldg(rewards + resp) - mu) / (sigma + (double)adv_eps));
 }
 
-template <bool KL, bool EXTRA>
+// VAR selects the score variants of the component ablations: 0 = the coefficient omega itself; 1 = chi_t r_t
+// replaced by 1 in the policy contribution; 2 = the advantage-only signal m_t A.
+template <bool KL, bool EXTRA, int VAR>
 __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid_constant__ CoeffArgs a)
 {
     const int64_t tile = blockIdx.x;
@@ -147,9 +149,14 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
             r[i] = expf(s[i] - o[i]);
             const bool c = pos ? (r[i] <= hi) : (r[i] >= lo);
             chi |= (uint32_t)c << (8 * i);
-            float v = (m && c) ? coef * r[i] : 0.0f;
-            if (KL && m)
-                v += kl * (-expm1f(rf[i] - s[i]));
+            float v;
+            if (VAR == 2) {
+                v = m ? A : 0.0f;
+            } else {
+                v = (VAR == 1) ? (m ? coef : 0.0f) : ((m && c) ? coef * r[i] : 0.0f);
+                if (KL && m)
+                    v += kl * (-expm1f(rf[i] - s[i]));
+            }
             w[i] = v;
         }
         const int64_t k = rowbase + t0[j];
@@ -322,12 +329,13 @@ extern "C" int hilore_mask_count(const uint8_t *mask, int64_t n, int64_t *count,
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
 }
 
-extern "C" int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
-                                  int64_t n_rows, int64_t T, const float *logp_new, const float *logp_old,
-                                  const float *logp_ref, const uint8_t *mask, int64_t N_norm,
-                                  const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps,
-                                  float *adv_out, float *omega, float *ratio, uint8_t *clip_mask, void *stream)
+static int launch_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset, int64_t n_rows,
+                         int64_t T, const float *logp_new, const float *logp_old, const float *logp_ref, const uint8_t *mask,
+                         int64_t N_norm, const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps, int variant,
+                         float *adv_out, float *omega, float *ratio, uint8_t *clip_mask, void *stream)
 {
+    if (variant < 0 || variant > 2)
+        return HILORE_INVALID_ARG;
     if (rewards == nullptr || n_resp_total < 0 || G <= 0 || resp_offset < 0 || n_rows < 0 || T < 0)
         return HILORE_INVALID_ARG;
     if (n_resp_total % G != 0 || resp_offset + n_rows > n_resp_total || T % 4 != 0)
@@ -371,11 +379,37 @@ extern "C" int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, in
     a.tiles_per_row = (int)tpr;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool kl = beta != 0.0f, extra = (ratio != nullptr) || (clip_mask != nullptr);
-    if (kl && extra) grpo_coeffs_kernel<true, true><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
-    else if (kl) grpo_coeffs_kernel<true, false><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
-    else if (extra) grpo_coeffs_kernel<false, true><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
-    else grpo_coeffs_kernel<false, false><<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
+    void (*kernel)(CoeffArgs) = nullptr;
+#define HILORE_PICK(V)                                                                                                  \
+    kernel = kl ? (extra ? grpo_coeffs_kernel<true, true, V> : grpo_coeffs_kernel<true, false, V>)                      \
+                : (extra ? grpo_coeffs_kernel<false, true, V> : grpo_coeffs_kernel<false, false, V>)
+    if (variant == 0) { HILORE_PICK(0); }
+    else if (variant == 1) { HILORE_PICK(1); }
+    else { HILORE_PICK(2); }
+#undef HILORE_PICK
+    kernel<<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
+
+extern "C" int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                                  int64_t n_rows, int64_t T, const float *logp_new, const float *logp_old,
+                                  const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                                  const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps,
+                                  float *adv_out, float *omega, float *ratio, uint8_t *clip_mask, void *stream)
+{
+    return launch_coeffs(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask, N_norm,
+                         N_norm_dev, clip_eps, beta, adv_eps, 0, adv_out, omega, ratio, clip_mask, stream);
+}
+
+extern "C" int hilore_grpo_coeffs_variant(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                                          int64_t n_rows, int64_t T, const float *logp_new, const float *logp_old,
+                                          const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                                          const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps,
+                                          int32_t variant, float *adv_out, float *omega, float *ratio, uint8_t *clip_mask,
+                                          void *stream)
+{
+    return launch_coeffs(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask, N_norm,
+                         N_norm_dev, clip_eps, beta, adv_eps, variant, adv_out, omega, ratio, clip_mask, stream);
 }
 
 extern "C" size_t hilore_workspace_bytes(int32_t U, int64_t n_tok)

@@ -73,6 +73,31 @@ def coeffs_point(log2_slots, reps, G=16, T=1024):
             "gbs": 13 * slots / t / 1e6}
 
 
+def diagnostics_point(log2_slots, reps, G=16, T=1024):
+    """The omega diagnostics (cause counts + exact top-decile share) over one record of coefficients."""
+    n_resp = max(G, (1 << log2_slots) // T)
+    slots = n_resp * T
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(2)
+    lp = torch.randn((n_resp, T), generator=gen, device="cuda") * 0.5 - 1.5
+    lo = lp + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.15
+    mask = (torch.rand((n_resp, T), generator=gen, device="cuda") < 0.8).to(torch.uint8)
+    rewards = (torch.rand(n_resp, generator=gen, device="cuda") < 0.5).float()
+    adv = torch.empty(n_resp, device="cuda")
+    omega, ratio = torch.empty_like(lp), torch.empty_like(lp)
+    api.hilore_grpo_coeffs(rewards, n_resp, G, 0, n_resp, T, lp, lo, None, mask, slots, None, 0.2, 0.0, 1e-6, adv, omega,
+                           ratio, None)
+    nws = api.hilore_omega_diagnostics_workspace_bytes()
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    counts = torch.zeros(5, dtype=torch.int64, device="cuda")
+    share, total = torch.zeros(1, dtype=torch.float64, device="cuda"), torch.zeros(1, dtype=torch.float64, device="cuda")
+    fn = lambda: api.hilore_omega_diagnostics(adv, ratio, mask, omega, n_resp, T, 0.2, counts, share, total, ws, nws)
+    t = _time([fn], reps)
+    # bytes the four sweeps read: 9 (ratio, mask, omega) + 3 x 5 (mask, omega) per slot
+    return {"kernel": "omega_diagnostics", "slots": slots, "us": t * 1e3, "slots_per_s": slots / t * 1e3,
+            "gbs": 24 * slots / t / 1e6, "zero_omega_fraction": counts[3].item() / slots, "top_decile_share": share.item()}
+
+
 def allocate_point(U, reps, N=1024):
     """The DP allocator on the paper's grid: U units, synthetic utilities / memory costs / risks."""
     import numpy as np
@@ -121,6 +146,8 @@ def main():
     if not a.no_coeffs:
         for ls in range(16, 25):
             print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
+        for ls in (20, 24, 27):
+            print(json.dumps(diagnostics_point(ls, max(3, a.reps // 4))), flush=True)
         for U in (36, 84):
             print(json.dumps(allocate_point(U, max(3, a.reps // 4))), flush=True)
 
