@@ -228,3 +228,28 @@ def omega_diagnostics(adv_rows, ratio, mask, omega, clip_eps=0.2):
                                        _p(omega, np.float32), C.c_int64(n_rows), C.c_int64(T), C.c_float(clip_eps),
                                        _p(counts, np.int64), C.byref(share), C.byref(total)))
     return counts, float(share.value), float(total.value)
+
+
+def grpo_coeffs_packed(adv_seq, cu_seqlens, logp_new, logp_old, logp_ref, mask, N_norm=0, clip_eps=0.2, beta=0.0):
+    """Packed layout: adv_seq [n_seq], cu_seqlens int32 [n_seq + 1], per-token arrays [n_tok]."""
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    n_seq, n_tok = len(cu) - 1, int(cu[-1])
+    adv_seq = np.ascontiguousarray(adv_seq, dtype=np.float32)
+    omega, ratio, chi = np.empty(n_tok, np.float32), np.empty(n_tok, np.float32), np.empty(n_tok, np.uint8)
+    _check(lib().orc_grpo_coeffs_packed(_p(adv_seq, np.float32), _p(cu, np.int32), C.c_int64(n_seq),
+                                        _p(logp_new, np.float32), _p(logp_old, np.float32), _p(logp_ref, np.float32),
+                                        _p(mask, np.uint8), C.c_int64(N_norm), C.c_float(clip_eps), C.c_float(beta),
+                                        _p(omega, np.float32), _p(ratio, np.float32), _p(chi, np.uint8)))
+    return omega, ratio, chi
+
+
+def unit_exposure_packed(omega, mask, cu_seqlens, rms, row_shift=0, eps_alpha=1e-8):
+    cu = np.ascontiguousarray(cu_seqlens, dtype=np.int32)
+    U, rms_ld = rms.shape
+    out = np.empty(U, np.float32)
+    sw = np.zeros(1, np.float32)
+    _check(lib().orc_unit_exposure_packed(_p(omega, np.float32), _p(mask, np.uint8), _p(cu, np.int32),
+                                          C.c_int64(len(cu) - 1), _p(rms, np.float32), C.c_int32(U), C.c_int64(rms_ld),
+                                          C.c_int32(row_shift), C.c_float(eps_alpha), _p(out, np.float32),
+                                          _p(sw, np.float32)))
+    return out, float(sw[0])

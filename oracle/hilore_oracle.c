@@ -35,6 +35,9 @@
  *   orc_grpo_coeffs_variant, orc_omega_diagnostics   hand-worked record, identities of Remark 1 (beta = 0:
  *                         zero-omega slots = padding + zero-advantage + clipped), NumPy sort for the
  *                         top-decile share, closed forms for uniform / one-hot |omega|
+ *   orc_grpo_coeffs_packed, orc_unit_exposure_packed   the dense functions above on the same tokens laid
+ *                         out with padding (every valid token equal, bit for bit), hand-worked two-sequence
+ *                         record, zero-length sequences, first-token rule of row_shift
  *   orc_allocate          the paper's allocator (knapsack DP on the conservative grid): exhaustive
  *                         enumeration of all 3^U assignments of the discretised problem, the
  *                         feasibility guarantee of upward rounding, the tie rules and the
@@ -607,6 +610,97 @@ double orc_fit_kappa(const double *x, const double *y, int64_t n)
         return 0.0;
     double k = sxy / sxx;
     return k > 0.0 ? k : 0.0;
+}
+
+/* ------------------------------------------------ packed (padding-removed) layout */
+/* The padding-removal execution setting of the paper's DSR-sub configuration: the sequences of a microbatch
+ * (prompt followed by response, no padding slots) lie back to back; sequence i owns tokens
+ * cu_seqlens[i] .. cu_seqlens[i+1]-1 and carries the advantage of response i.  The arithmetic per token is
+ * that of orc_grpo_coeffs; the mask now excludes prompt tokens only. */
+int orc_grpo_coeffs_packed(const float *adv, const int32_t *cu_seqlens, int64_t n_seq, const float *logp_new,
+                           const float *logp_old, const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                           float clip_eps, float beta, float *omega, float *ratio, uint8_t *clip_mask)
+{
+    if (!adv || !cu_seqlens || n_seq < 0 || !logp_new || !logp_old || !mask || !omega)
+        return ORC_INVALID;
+    if (beta != 0.0f && !logp_ref)
+        return ORC_INVALID;
+    if (cu_seqlens[0] != 0)
+        return ORC_SHAPE;
+    for (int64_t i = 0; i < n_seq; ++i)
+        if (cu_seqlens[i + 1] < cu_seqlens[i])
+            return ORC_SHAPE;
+    const int64_t n_tok = cu_seqlens[n_seq];
+    int64_t N = N_norm;
+    if (N <= 0) {
+        N = 0;
+        for (int64_t k = 0; k < n_tok; ++k) N += mask[k] ? 1 : 0;
+    }
+    if (N <= 0)
+        return ORC_ZERO_NORM;
+    const float hi = 1.0f + clip_eps, lo = 1.0f - clip_eps;
+    for (int64_t i = 0; i < n_seq; ++i) {
+        const float A = adv[i];
+        for (int64_t k = cu_seqlens[i]; k < cu_seqlens[i + 1]; ++k) {
+            double r = exp((double)logp_new[k] - (double)logp_old[k]);
+            float r32 = (float)r;
+            int chi = (A >= 0.0f && r32 <= hi) || (A < 0.0f && r32 >= lo);
+            double m = mask[k] ? 1.0 : 0.0;
+            double w = -(m / (double)N) * (chi ? 1.0 : 0.0) * r * (double)A;
+            if (beta != 0.0f)
+                w += (double)beta * (m / (double)N) * (1.0 - exp((double)logp_ref[k] - (double)logp_new[k]));
+            omega[k] = (float)w;
+            if (ratio) ratio[k] = r32;
+            if (clip_mask) clip_mask[k] = (uint8_t)chi;
+        }
+    }
+    return ORC_OK;
+}
+
+/* orc_unit_exposure on the packed layout: the activation row of token k is k - row_shift, taken only when it
+ * lies inside the token's own sequence. */
+int orc_unit_exposure_packed(const float *omega, const uint8_t *mask, const int32_t *cu_seqlens, int64_t n_seq,
+                             const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift, float eps_alpha,
+                             float *exposure, float *sum_abs_omega)
+{
+    if (!omega || !mask || !cu_seqlens || !row_rms || !exposure || n_seq < 0 || U < 0)
+        return ORC_INVALID;
+    if (row_shift < 0 || row_shift > 1)
+        return ORC_INVALID;
+    const int64_t n_tok = cu_seqlens[n_seq];
+    if (rms_ld < n_tok)
+        return ORC_SHAPE;
+    int64_t cnt = 0;
+    double sw = 0.0;
+    for (int64_t k = 0; k < n_tok; ++k)
+        if (mask[k]) {
+            ++cnt;
+            sw += fabs((double)omega[k]);
+        }
+    if (sum_abs_omega)
+        *sum_abs_omega = (float)sw;
+    for (int32_t u = 0; u < U; ++u) {
+        const float *a = row_rms + (int64_t)u * rms_ld;
+        if (cnt == 0) {
+            exposure[u] = 0.0f;
+            continue;
+        }
+        double abar = 0.0;
+        for (int64_t i = 0; i < n_seq; ++i)
+            for (int64_t k = cu_seqlens[i]; k < cu_seqlens[i + 1]; ++k)
+                if (mask[k] && k - row_shift >= cu_seqlens[i])
+                    abar += (double)a[k - row_shift];
+        abar /= (double)cnt;
+        double E = 0.0;
+        for (int64_t i = 0; i < n_seq; ++i)
+            for (int64_t k = cu_seqlens[i]; k < cu_seqlens[i + 1]; ++k)
+                if (mask[k] && k - row_shift >= cu_seqlens[i]) {
+                    double alpha = ((double)a[k - row_shift] + (double)eps_alpha) / (abar + (double)eps_alpha);
+                    E += fabs((double)omega[k]) * alpha;
+                }
+        exposure[u] = (float)E;
+    }
+    return ORC_OK;
 }
 
 /* ------------------------------------------------ diagnostics and score variants on omega */

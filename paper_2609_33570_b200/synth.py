@@ -113,6 +113,46 @@ def rollout(seed: int, P: int, G: int, T: int, *, rewards: str = "bernoulli",
     return Rollout(P, G, T, R, logp_new, logp_old, logp_ref, mask, L)
 
 
+@dataclass
+class PackedRollout:
+    """A microbatch in the padding-removed layout: sequence i = prompt tokens then the valid response tokens of
+    row `rows[i]` of a dense Rollout; tokens of all sequences back to back."""
+    cu_seqlens: np.ndarray  # [n_seq + 1] int32
+    rows: np.ndarray        # [n_seq] int64, response index in the dense rollout
+    logp_new: np.ndarray    # [n_tok] fp32
+    logp_old: np.ndarray
+    logp_ref: np.ndarray
+    mask: np.ndarray        # [n_tok] uint8, 1 = generated response token
+    dense_t: np.ndarray     # [n_tok] int64: response slot t of the token in the dense layout, -1 for prompt tokens
+
+    @property
+    def n_tok(self) -> int:
+        return int(self.cu_seqlens[-1])
+
+
+def pack_rollout(ro: Rollout, seed: int, rows=None, max_prompt: int = 64, min_prompt: int = 1) -> PackedRollout:
+    """Re-lay rows `rows` (default: all) of a dense rollout without padding, each behind a prompt of random length
+    U{min_prompt..max_prompt} whose log-probabilities are drawn like the response's (they are masked out)."""
+    rng = np.random.default_rng(np.random.SeedSequence([seed, 77]))
+    rows = np.arange(ro.n_resp, dtype=np.int64) if rows is None else np.asarray(rows, dtype=np.int64)
+    plen = rng.integers(min_prompt, max_prompt + 1, size=len(rows), dtype=np.int64)
+    lens = plen + ro.lengths[rows]
+    cu = np.zeros(len(rows) + 1, dtype=np.int64)
+    np.cumsum(lens, out=cu[1:])
+    n_tok = int(cu[-1])
+    out = {k: np.empty(n_tok, np.float32) for k in ("logp_new", "logp_old", "logp_ref")}
+    mask = np.zeros(n_tok, np.uint8)
+    dense_t = np.full(n_tok, -1, np.int64)
+    for j, i in enumerate(rows):
+        a, b, L = int(cu[j]), int(cu[j] + plen[j]), int(ro.lengths[i])
+        for k in out:
+            out[k][a:b] = (rng.standard_normal(b - a, dtype=np.float32) * np.float32(0.5) - np.float32(1.5))
+            out[k][b:b + L] = getattr(ro, k)[i, :L]
+        mask[b:b + L] = ro.mask[i, :L]
+        dense_t[b:b + L] = np.arange(L)
+    return PackedRollout(cu.astype(np.int32), rows, out["logp_new"], out["logp_old"], out["logp_ref"], mask, dense_t)
+
+
 # Unit widths (attention input, MLP input, MLP intermediate) of the decoder shapes the configs name.
 UNIT_WIDTHS = {
     "0.5B": (896, 896, 4864),
