@@ -111,6 +111,35 @@ int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, in
                        float *omega, float *ratio, uint8_t *clip_mask, void *stream);
 
 /*
+ * The coefficient and exposure passes on the packed (padding-removed) layout of the paper's DSR-sub execution
+ * setting (Table "execution-configurations": "padding removal").  The sequences of a microbatch -- prompt
+ * followed by the generated response, no padding slots -- lie back to back: sequence i (response
+ * resp_offset + i of the rollout batch) owns tokens cu_seqlens[i] .. cu_seqlens[i+1]-1; the activation
+ * tensors of the microbatch have one row per packed token.  Arithmetic per token exactly as in
+ * hilore_grpo_coeffs / hilore_unit_exposure; mask = 1 on generated response tokens, 0 on prompt tokens.
+ *
+ *   cu_seqlens   [n_seq + 1] int32 on the device, cu_seqlens[0] = 0, non-decreasing (empty sequences allowed),
+ *                cu_seqlens[n_seq] = n_tok.  The contents are the caller's responsibility (they are not read on
+ *                the host); whatever they hold, no kernel indexes outside [0, n_seq] or [0, n_tok).
+ *   logp_*, omega, ratio [n_tok] fp32, 16-byte aligned;  mask, clip_mask [n_tok] u8, 4-byte aligned; n_tok need
+ *                not be a multiple of 4 (n_tok < 2^31).
+ *   adv_out      [n_seq] fp32, REQUIRED here: the per-sequence advantages are written by a first launch and read
+ *                by the token kernel (2 launches).
+ *   Exposure: the activation row of token k is k - row_shift; with row_shift = 1 a token whose source row
+ *   would fall before the start of its own sequence has no activation term (it still counts in |T_b|).
+ *   Other arguments, status codes and workspace as in the dense calls.
+ */
+int hilore_grpo_coeffs_packed(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                              int64_t n_seq, const int32_t *cu_seqlens, int64_t n_tok, const float *logp_new,
+                              const float *logp_old, const float *logp_ref, const uint8_t *mask, int64_t N_norm,
+                              const int64_t *N_norm_dev, float clip_eps, float beta, float adv_eps, float *adv_out,
+                              float *omega, float *ratio, uint8_t *clip_mask, void *stream);
+int hilore_unit_exposure_packed(const float *omega, const uint8_t *mask, int64_t n_tok, const int32_t *cu_seqlens,
+                                int64_t n_seq, const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
+                                size_t workspace_bytes, void *stream);
+
+/*
  * Score variants of the component ablations (paragraph "Component ablations"): hilore_grpo_coeffs with one
  * more argument.  variant 0: omega as above.  variant 1 ("removing ratio/clipping"): chi_t r_t replaced by 1 in
  * the policy contribution, omega_t = -(m_t / N) A + beta (m_t / N)(1 - exp(s_ref - s)).  variant 2: the

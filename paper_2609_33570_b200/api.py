@@ -26,7 +26,8 @@ EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "h
            "hilore_plan_apply", "hilore_unit_exposure_static", "hilore_static_scratch_bytes",
            "hilore_allocate", "hilore_allocate_workspace_bytes", "hilore_risk_budget",
            "hilore_relative_error", "hilore_relative_error_workspace_bytes", "hilore_fit_kappa",
-           "hilore_grpo_coeffs_variant", "hilore_omega_diagnostics", "hilore_omega_diagnostics_workspace_bytes")
+           "hilore_grpo_coeffs_variant", "hilore_omega_diagnostics", "hilore_omega_diagnostics_workspace_bytes",
+           "hilore_grpo_coeffs_packed", "hilore_unit_exposure_packed")
 
 
 class HiloreUnit(C.Structure):
@@ -83,6 +84,9 @@ def lib() -> C.CDLL:
         _lib.hilore_fit_kappa.argtypes = [vp, vp, i64]
         _lib.hilore_grpo_coeffs_variant.argtypes = [vp, i64, i32, i64, i64, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32, i32,
                                                     vp, vp, vp, vp, vp]
+        _lib.hilore_grpo_coeffs_packed.argtypes = [vp, i64, i32, i64, i64, vp, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32,
+                                                   vp, vp, vp, vp, vp]
+        _lib.hilore_unit_exposure_packed.argtypes = [vp, vp, i64, vp, i64, vp, i32, i64, i32, f32, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_omega_diagnostics.argtypes = [vp, vp, vp, vp, i64, i64, f32, vp, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_omega_diagnostics_workspace_bytes.restype = C.c_size_t
         _lib.hilore_omega_diagnostics_workspace_bytes.argtypes = []
@@ -145,6 +149,24 @@ def hilore_grpo_coeffs_variant(rewards, n_resp_total, G, resp_offset, n_rows, T,
                                           clip_eps, beta, adv_eps, variant, _ptr(adv_out), _ptr(omega), _ptr(ratio),
                                           _ptr(clip_mask), _stream(stream))
     return _check(st, "hilore_grpo_coeffs_variant", check)
+
+
+def hilore_grpo_coeffs_packed(rewards, n_resp_total, G, resp_offset, n_seq, cu_seqlens, n_tok, logp_new, logp_old,
+                              logp_ref, mask, N_norm, N_norm_dev, clip_eps, beta, adv_eps, adv_out, omega, ratio,
+                              clip_mask, stream=None, check=True):
+    st = lib().hilore_grpo_coeffs_packed(_ptr(rewards), n_resp_total, G, resp_offset, n_seq, _ptr(cu_seqlens), n_tok,
+                                         _ptr(logp_new), _ptr(logp_old), _ptr(logp_ref), _ptr(mask), N_norm,
+                                         _ptr(N_norm_dev), clip_eps, beta, adv_eps, _ptr(adv_out), _ptr(omega),
+                                         _ptr(ratio), _ptr(clip_mask), _stream(stream))
+    return _check(st, "hilore_grpo_coeffs_packed", check)
+
+
+def hilore_unit_exposure_packed(omega, mask, n_tok, cu_seqlens, n_seq, row_rms, U, rms_ld, row_shift, eps_alpha,
+                                exposure, sum_abs_omega, workspace, workspace_bytes, stream=None, check=True):
+    st = lib().hilore_unit_exposure_packed(_ptr(omega), _ptr(mask), n_tok, _ptr(cu_seqlens), n_seq, _ptr(row_rms), U,
+                                           rms_ld, row_shift, eps_alpha, _ptr(exposure), _ptr(sum_abs_omega),
+                                           _ptr(workspace), workspace_bytes, _stream(stream))
+    return _check(st, "hilore_unit_exposure_packed", check)
 
 
 def hilore_omega_diagnostics_workspace_bytes():

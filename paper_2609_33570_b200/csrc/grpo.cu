@@ -58,10 +58,15 @@ constexpr int kCoeffThreads = 128;
 constexpr int kCoeffVec = 2;                                  // float4 groups per thread
 constexpr int kCoeffTile = kCoeffThreads * kCoeffVec * 4;     // 1024 slots of one response per CTA
 
-// Advantage of response `resp`, from the G rewards of its prompt group, in fp64 (one warp).
-__device__ float group_advantage(const float *rewards, int64_t resp, int G, float adv_eps, int lane)
+// Mean and population standard deviation of the G rewards of one prompt group, in fp64 (one warp; every lane
+// returns the same values).  `equal` is set when all G rewards are the same number.
+struct GroupStats {
+    double mu, sigma;
+    bool equal;
+};
+
+__device__ __forceinline__ GroupStats group_stats(const float *R, int G, int lane)
 {
-    const float *R = rewards + (resp / G) * G;
     float lo = INFINITY, hi = -INFINITY;
     double sum = 0.0;
     for (int j = lane; j < G; j += 32) {
@@ -76,17 +81,33 @@ __device__ float group_advantage(const float *rewards, int64_t resp, int G, floa
         hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
     }
     sum = warp_sum(sum);
-    if (lo == hi)
-        return 0.0f; // equal-reward group: exactly zero, whatever the rounding of the mean
-    const double mu = sum / (double)G;
+    GroupStats g;
+    g.equal = lo == hi;
+    g.mu = sum / (double)G;
+    g.sigma = 0.0;
+    if (g.equal)
+        return g;
     double var = 0.0;
     for (int j = lane; j < G; j += 32) {
-        const double d = (double)__ldg(R + j) - mu;
+        const double d = (double)__ldg(R + j) - g.mu;
         var += d * d;
     }
     var = warp_sum(var) / (double)G;
-    const double sigma = sqrt(var);
-    return (float)(((double)__ldg(rewards + resp) - mu) / (sigma + (double)adv_eps));
+    g.sigma = sqrt(var);
+    return g;
+}
+
+// Advantage of a response with reward `r`: exactly zero in an equal-reward group, whatever the rounding of the mean.
+__device__ __forceinline__ float advantage_of(const GroupStats &g, float r, float adv_eps)
+{
+    return g.equal ? 0.0f : (float)(((double)r - g.mu) / (g.sigma + (double)adv_eps));
+}
+
+// Advantage of response `resp`, from the G rewards of its prompt group (one warp).
+__device__ float group_advantage(const float *rewards, int64_t resp, int G, float adv_eps, int lane)
+{
+    const GroupStats g = group_stats(rewards + (resp / G) * G, G, lane);
+    return advantage_of(g, __ldg(rewards + resp), adv_eps);
 }
 
 // VAR selects the score variants of the component ablations: 0 = the coefficient omega itself; 1 = chi_t r_t
@@ -168,6 +189,175 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
     }
 }
 
+// ------------------------------------------------------------------ coefficients, packed layout
+// Sequences lie back to back (no padding slots); sequence i owns tokens cu[i] .. cu[i+1]-1.
+// Index of the sequence that owns token k: the largest i < n_seq with cu[i] <= k.  Bounded for any contents.
+__device__ __forceinline__ int owner_sequence(const int32_t *cu, int n_seq, int64_t k, int lo = 0)
+{
+    int hi = n_seq; // invariant: cu[lo] <= k (cu[0] = 0), answer in [lo, hi)
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((int64_t)__ldg(cu + mid) <= k) lo = mid;
+        else hi = mid;
+    }
+    return lo;
+}
+
+// The same search by one whole warp: 32 probes per step, so a table of a million sequences takes four dependent
+// loads instead of twenty.  All lanes return the answer.
+__device__ __forceinline__ int owner_sequence_warp(const int32_t *cu, int n_seq, int64_t k, int lane)
+{
+    int lo = 0, hi = n_seq;
+    while (hi - lo > 1) {
+        const int64_t span = hi - lo;
+        const int p = lo + (int)((span * (lane + 1)) / 33); // lo <= p < hi
+        const int nle = __popc(__ballot_sync(0xFFFFFFFFu, (int64_t)__ldg(cu + p) <= k));
+        const int new_lo = lo + (int)((span * nle) / 33);
+        const int new_hi = nle < 32 ? lo + (int)((span * (nle + 1)) / 33) : hi;
+        lo = new_lo;
+        hi = new_hi;
+    }
+    return lo;
+}
+
+// One warp per prompt group that meets the microbatch: the statistics once, then the members' advantages.
+__global__ void __launch_bounds__(128) packed_advantage_kernel(const float *rewards, int64_t resp_offset, int64_t n_seq, int G,
+                                                                float adv_eps, float *adv)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t g = resp_offset / G + (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (g * G >= resp_offset + n_seq) return;
+    const GroupStats st = group_stats(rewards + g * G, G, lane);
+    for (int j = lane; j < G; j += 32) {
+        const int64_t resp = g * G + j;
+        if (resp >= resp_offset && resp < resp_offset + n_seq)
+            adv[resp - resp_offset] = advantage_of(st, __ldg(rewards + resp), adv_eps);
+    }
+}
+
+struct PackedArgs {
+    const int32_t *cu;
+    int n_seq;
+    int64_t n_tok;
+    const float *adv, *logp_new, *logp_old, *logp_ref;
+    const uint8_t *mask;
+    int64_t N_norm;
+    const long long *N_norm_dev;
+    float clip_eps, beta;
+    float *omega, *ratio;
+    uint8_t *clip_mask;
+};
+
+template <bool KL, bool EXTRA>
+__global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_packed_kernel(const __grid_constant__ PackedArgs a)
+{
+    const int tid = threadIdx.x;
+    float4 sn[kCoeffVec], so[kCoeffVec], sr[kCoeffVec];
+    uint32_t mk[kCoeffVec];
+    int64_t k0[kCoeffVec];
+    int cnt[kCoeffVec];
+#pragma unroll
+    for (int j = 0; j < kCoeffVec; ++j) {
+        k0[j] = (int64_t)blockIdx.x * kCoeffTile + (int64_t)(j * kCoeffThreads + tid) * 4;
+        const int64_t left = a.n_tok - k0[j];
+        cnt[j] = left >= 4 ? 4 : (left > 0 ? (int)left : 0);
+        if (cnt[j] == 4) {
+            sn[j] = __ldcs(reinterpret_cast<const float4 *>(a.logp_new + k0[j]));
+            so[j] = __ldcs(reinterpret_cast<const float4 *>(a.logp_old + k0[j]));
+            if (KL) sr[j] = __ldcs(reinterpret_cast<const float4 *>(a.logp_ref + k0[j]));
+            mk[j] = __ldcs(reinterpret_cast<const unsigned int *>(a.mask + k0[j]));
+        } else if (cnt[j] > 0) { // ragged end of the microbatch: element by element
+            float tn[4] = {0, 0, 0, 0}, to[4] = {0, 0, 0, 0}, tr[4] = {0, 0, 0, 0};
+            uint32_t m = 0;
+            for (int i = 0; i < cnt[j]; ++i) {
+                tn[i] = a.logp_new[k0[j] + i];
+                to[i] = a.logp_old[k0[j] + i];
+                if (KL) tr[i] = a.logp_ref[k0[j] + i];
+                m |= (uint32_t)(a.mask[k0[j] + i] != 0) << (8 * i);
+            }
+            sn[j] = make_float4(tn[0], tn[1], tn[2], tn[3]);
+            so[j] = make_float4(to[0], to[1], to[2], to[3]);
+            sr[j] = make_float4(tr[0], tr[1], tr[2], tr[3]);
+            mk[j] = m;
+        }
+    }
+    // the sequences that meet this tile: found once per CTA (two searches over the whole table, in parallel with
+    // the token loads), then each group searches that short range only
+    __shared__ int s_range[2];
+    __shared__ int64_t s_first_end;
+    __shared__ float s_first_adv;
+    if (tid < 64) {
+        const int64_t first = (int64_t)blockIdx.x * kCoeffTile;
+        const int64_t last = min(first + kCoeffTile, a.n_tok) - 1;
+        const int own = owner_sequence_warp(a.cu, a.n_seq, tid < 32 ? first : last, tid & 31);
+        if ((tid & 31) == 0) s_range[tid >> 5] = own;
+        if (tid == 0) { // most groups of a tile lie in its first sequence: its end and advantage go to shared memory
+            s_first_end = (int64_t)__ldg(a.cu + own + 1);
+            s_first_adv = __ldg(a.adv + own);
+        }
+    }
+    __syncthreads();
+    const int seq_first = s_range[0], seq_end = s_range[1] + 1;
+    const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
+    const double invN = N > 0 ? 1.0 / (double)N : 0.0;
+    const float kl = (float)((double)a.beta * invN);
+    const float hi = 1.0f + a.clip_eps, lo = 1.0f - a.clip_eps;
+
+#pragma unroll
+    for (int j = 0; j < kCoeffVec; ++j) {
+        if (cnt[j] == 0)
+            continue;
+        int seq = seq_first;
+        int64_t end = s_first_end;
+        float A = s_first_adv;
+        if (k0[j] >= end) {
+            seq = owner_sequence(a.cu, seq_end, k0[j], seq_first);
+            end = (int64_t)__ldg(a.cu + seq + 1);
+            A = __ldg(a.adv + seq);
+        }
+        float coef = (float)(-(double)A * invN);
+        const float s[4] = {sn[j].x, sn[j].y, sn[j].z, sn[j].w};
+        const float o[4] = {so[j].x, so[j].y, so[j].z, so[j].w};
+        const float rf[4] = {sr[j].x, sr[j].y, sr[j].z, sr[j].w};
+        float w[4], r[4];
+        uint32_t chi = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (k0[j] + i >= end && i < cnt[j]) { // the group crosses into the next non-empty sequence
+                while (seq + 1 < a.n_seq && k0[j] + i >= end) {
+                    ++seq;
+                    end = (int64_t)__ldg(a.cu + seq + 1);
+                }
+                A = __ldg(a.adv + seq);
+                coef = (float)(-(double)A * invN);
+            }
+            const bool m = ((mk[j] >> (8 * i)) & 0xFFu) != 0;
+            r[i] = expf(s[i] - o[i]);
+            const bool c = (A >= 0.0f) ? (r[i] <= hi) : (r[i] >= lo);
+            chi |= (uint32_t)c << (8 * i);
+            float v = (m && c) ? coef * r[i] : 0.0f;
+            if (KL && m)
+                v += kl * (-expm1f(rf[i] - s[i]));
+            w[i] = v;
+        }
+        if (cnt[j] == 4) {
+            __stcs(reinterpret_cast<float4 *>(a.omega + k0[j]), make_float4(w[0], w[1], w[2], w[3]));
+            if (EXTRA) {
+                if (a.ratio) __stcs(reinterpret_cast<float4 *>(a.ratio + k0[j]), make_float4(r[0], r[1], r[2], r[3]));
+                if (a.clip_mask) __stcs(reinterpret_cast<unsigned int *>(a.clip_mask + k0[j]), chi);
+            }
+        } else {
+            for (int i = 0; i < cnt[j]; ++i) {
+                a.omega[k0[j] + i] = w[i];
+                if (EXTRA) {
+                    if (a.ratio) a.ratio[k0[j] + i] = r[i];
+                    if (a.clip_mask) a.clip_mask[k0[j] + i] = (uint8_t)((chi >> (8 * i)) & 1u);
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------ exposure
 constexpr int kExpThreads = 256;
 constexpr int kExpTile = kExpThreads * 4; // slots per CTA
@@ -183,6 +373,8 @@ struct ExpArgs {
     int row_shift;
     double *part; // [(U + 1), ntiles, 2]
     int ntiles;
+    const int32_t *cu; // packed layout: sequence boundaries (else nullptr: rows of T slots)
+    int n_seq;
 };
 
 template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __grid_constant__ ExpArgs a)
@@ -228,7 +420,9 @@ template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_part
                 mk[i] = true;
                 wabs[i] = fabsf(a.omega[k]);
                 // a slot whose source row lies before the start of its response has no activation term
-                has[i] = a.row_shift == 0 || (k % a.T) >= a.row_shift;
+                if (a.row_shift == 0) has[i] = true;
+                else if (a.cu) has[i] = k - (int64_t)__ldg(a.cu + owner_sequence(a.cu, a.n_seq, k)) >= a.row_shift;
+                else has[i] = (k % a.T) >= a.row_shift;
             }
         }
     }
@@ -420,24 +614,23 @@ extern "C" size_t hilore_workspace_bytes(int32_t U, int64_t n_tok)
     return (size_t)(U + 1) * (size_t)(ntiles > 0 ? ntiles : 1) * 2 * sizeof(double);
 }
 
-extern "C" int hilore_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
-                                    const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
-                                    float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
-                                    size_t workspace_bytes, void *stream)
+static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T, int64_t n_tok,
+                           const int32_t *cu, int64_t n_seq, const float *row_rms, int32_t U, int64_t rms_ld,
+                           int32_t row_shift, float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
+                           size_t workspace_bytes, void *stream)
 {
-    if (n_rows < 0 || T < 0 || U < 0 || row_shift < 0 || row_shift > 1)
+    if (n_rows < 0 || T < 0 || n_tok < 0 || U < 0 || row_shift < 0 || row_shift > 1)
         return HILORE_INVALID_ARG;
     if (U == 0)
         return HILORE_OK;
     if (exposure == nullptr || row_rms == nullptr || workspace == nullptr)
         return HILORE_INVALID_ARG;
-    const int64_t n_tok = n_rows * T;
     if (n_tok > 0 && (omega == nullptr || mask == nullptr))
         return HILORE_INVALID_ARG;
     if (rms_ld < n_tok)
         return HILORE_SHAPE;
     if (!aligned(workspace, 16) || !aligned(omega, 4) || !aligned(row_rms, 4) || !aligned(exposure, 4) ||
-        !aligned(sum_abs_omega, 4))
+        !aligned(sum_abs_omega, 4) || !aligned(cu, 4))
         return HILORE_ALIGN;
     if (workspace_bytes < hilore_workspace_bytes(U, n_tok))
         return HILORE_WORKSPACE;
@@ -457,6 +650,8 @@ extern "C" int hilore_unit_exposure(const float *omega, const uint8_t *mask, int
     a.row_shift = row_shift;
     a.part = static_cast<double *>(workspace);
     a.ntiles = (int)ntiles64;
+    a.cu = cu;
+    a.n_seq = (int)n_seq;
     if (a.ntiles > 0) {
         const dim3 grid((unsigned)a.ntiles, (unsigned)((U + kExpUnits - 1) / kExpUnits));
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
@@ -467,6 +662,84 @@ extern "C" int hilore_unit_exposure(const float *omega, const uint8_t *mask, int
             return HILORE_CUDA;
     }
     exposure_final_kernel<<<(unsigned)U, 32, 0, st>>>(a.part, U, a.ntiles, eps_alpha, exposure, sum_abs_omega);
+    return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
+
+extern "C" int hilore_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
+                                    const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                    float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
+                                    size_t workspace_bytes, void *stream)
+{
+    if (n_rows < 0 || T < 0)
+        return HILORE_INVALID_ARG;
+    return launch_exposure(omega, mask, n_rows, T, n_rows * T, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha,
+                           exposure, sum_abs_omega, workspace, workspace_bytes, stream);
+}
+
+extern "C" int hilore_unit_exposure_packed(const float *omega, const uint8_t *mask, int64_t n_tok,
+                                           const int32_t *cu_seqlens, int64_t n_seq, const float *row_rms, int32_t U,
+                                           int64_t rms_ld, int32_t row_shift, float eps_alpha, float *exposure,
+                                           float *sum_abs_omega, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (n_tok < 0 || n_tok > 0x7FFFFFFF || n_seq < 0 || n_seq > 0x7FFFFFFE || (n_tok > 0 && (cu_seqlens == nullptr || n_seq == 0)))
+        return HILORE_INVALID_ARG;
+    return launch_exposure(omega, mask, 1, n_tok, n_tok, n_tok > 0 ? cu_seqlens : nullptr, n_seq, row_rms, U, rms_ld,
+                           row_shift, eps_alpha, exposure, sum_abs_omega, workspace, workspace_bytes, stream);
+}
+
+extern "C" int hilore_grpo_coeffs_packed(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
+                                         int64_t n_seq, const int32_t *cu_seqlens, int64_t n_tok, const float *logp_new,
+                                         const float *logp_old, const float *logp_ref, const uint8_t *mask,
+                                         int64_t N_norm, const int64_t *N_norm_dev, float clip_eps, float beta,
+                                         float adv_eps, float *adv_out, float *omega, float *ratio, uint8_t *clip_mask,
+                                         void *stream)
+{
+    if (rewards == nullptr || n_resp_total < 0 || G <= 0 || resp_offset < 0 || n_seq < 0 || n_tok < 0)
+        return HILORE_INVALID_ARG;
+    if (n_resp_total % G != 0 || resp_offset + n_seq > n_resp_total || n_tok > 0x7FFFFFFF || n_seq > 0x7FFFFFFE)
+        return HILORE_SHAPE;
+    if (beta != 0.0f && logp_ref == nullptr)
+        return HILORE_INVALID_ARG;
+    if (N_norm_dev == nullptr && N_norm <= 0)
+        return HILORE_ZERO_NORM;
+    if (n_seq == 0)
+        return n_tok == 0 ? HILORE_OK : HILORE_SHAPE;
+    if (cu_seqlens == nullptr || adv_out == nullptr)
+        return HILORE_INVALID_ARG;
+    if (n_tok > 0 && (logp_new == nullptr || logp_old == nullptr || mask == nullptr || omega == nullptr))
+        return HILORE_INVALID_ARG;
+    if (!aligned(logp_new, 16) || !aligned(logp_old, 16) || !aligned(logp_ref, 16) || !aligned(omega, 16) ||
+        !aligned(ratio, 16) || !aligned(mask, 4) || !aligned(clip_mask, 4) || !aligned(rewards, 4) ||
+        !aligned(adv_out, 4) || !aligned(N_norm_dev, 8) || !aligned(cu_seqlens, 4))
+        return HILORE_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t n_groups = (resp_offset + n_seq + G - 1) / G - resp_offset / G;
+    packed_advantage_kernel<<<(unsigned)((n_groups + 3) / 4), 128, 0, st>>>(rewards, resp_offset, n_seq, G, adv_eps, adv_out);
+    if (cudaGetLastError() != cudaSuccess)
+        return HILORE_CUDA;
+    if (n_tok == 0)
+        return HILORE_OK;
+    PackedArgs a{};
+    a.cu = cu_seqlens;
+    a.n_seq = (int)n_seq;
+    a.n_tok = n_tok;
+    a.adv = adv_out;
+    a.logp_new = logp_new;
+    a.logp_old = logp_old;
+    a.logp_ref = (beta != 0.0f) ? logp_ref : nullptr;
+    a.mask = mask;
+    a.N_norm = N_norm;
+    a.N_norm_dev = reinterpret_cast<const long long *>(N_norm_dev);
+    a.clip_eps = clip_eps;
+    a.beta = beta;
+    a.omega = omega;
+    a.ratio = ratio;
+    a.clip_mask = clip_mask;
+    const int64_t tiles = (n_tok + kCoeffTile - 1) / kCoeffTile;
+    const bool kl = beta != 0.0f, extra = (ratio != nullptr) || (clip_mask != nullptr);
+    void (*kernel)(PackedArgs) = kl ? (extra ? grpo_coeffs_packed_kernel<true, true> : grpo_coeffs_packed_kernel<true, false>)
+                                    : (extra ? grpo_coeffs_packed_kernel<false, true> : grpo_coeffs_packed_kernel<false, false>);
+    kernel<<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
 }
 

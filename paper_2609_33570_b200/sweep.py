@@ -73,6 +73,34 @@ def coeffs_point(log2_slots, reps, G=16, T=1024):
             "gbs": 13 * slots / t / 1e6}
 
 
+def coeffs_packed_point(log2_tokens, reps, G=8, mean_len=2048):
+    """The coefficient kernel on the packed layout: sequences of U{mean_len/2 .. 3 mean_len/2} tokens back to back."""
+    import numpy as np
+    n_tok = 1 << log2_tokens
+    rng = np.random.default_rng(log2_tokens)
+    lens = rng.integers(mean_len // 2, 3 * mean_len // 2 + 1, size=2 * n_tok // mean_len + 8)
+    ends = np.cumsum(lens)
+    ends = ends[: int(np.searchsorted(ends, n_tok)) + 1]
+    ends[-1] = n_tok
+    ends = np.concatenate([ends, np.full((-len(ends)) % G, n_tok)])      # empty sequences fill the last group
+    n_seq = len(ends)
+    cu = torch.from_numpy(np.concatenate([[0], ends]).astype(np.int32)).cuda()
+    pool = max(1, min(8, -(-3 * L2_BYTES // (n_tok * 13))))
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(3)
+    lp = [torch.randn(n_tok, generator=gen, device="cuda") * 0.5 - 1.5 for _ in range(pool)]
+    lo = [x + torch.randn(n_tok, generator=gen, device="cuda") * 0.05 for x in lp]
+    mask = (torch.rand(n_tok, generator=gen, device="cuda") < 0.75).to(torch.uint8)
+    rewards = (torch.rand(n_seq, generator=gen, device="cuda") < 0.5).float()
+    adv = torch.empty(n_seq, device="cuda")
+    omega = [torch.empty_like(x) for x in lp]
+    fns = [lambda i=i: api.hilore_grpo_coeffs_packed(rewards, n_seq, G, 0, n_seq, cu, n_tok, lp[i], lo[i], None, mask, n_tok,
+                                                     None, 0.2, 0.0, 1e-6, adv, omega[i], None, None) for i in range(pool)]
+    t = _time(fns, reps)
+    return {"kernel": "grpo_coeffs_packed", "tokens": n_tok, "n_seq": n_seq, "pool": pool, "us": t * 1e3,
+            "tokens_per_s": n_tok / t * 1e3, "gbs": 13 * n_tok / t / 1e6}
+
+
 def diagnostics_point(log2_slots, reps, G=16, T=1024):
     """The omega diagnostics (cause counts + exact top-decile share) over one record of coefficients."""
     n_resp = max(G, (1 << log2_slots) // T)
@@ -146,6 +174,8 @@ def main():
     if not a.no_coeffs:
         for ls in range(16, 25):
             print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
+        for ls in (15, 20, 24, 27):
+            print(json.dumps(coeffs_packed_point(ls, a.reps)), flush=True)
         for ls in (20, 24, 27):
             print(json.dumps(diagnostics_point(ls, max(3, a.reps // 4))), flush=True)
         for U in (36, 84):

@@ -1,0 +1,127 @@
+"""Parity of the packed-layout coefficient and exposure calls with the oracle (fp32 within 1e-5 relative; the clip
+indicator exact away from the clip bounds), and equality with the dense kernels on the same tokens."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_33570_b200 import api, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-5
+
+
+def dev_i32(a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+
+
+def packed_gpu(ro, pk, beta=0.0, N=None, resp_offset=0, n_on_device=False):
+    n_seq, n_tok = len(pk.rows), pk.n_tok
+    adv, omega = G.Guarded(max(n_seq, 1) * 4), G.Guarded(n_tok * 4)
+    ratio, chi = G.Guarded(n_tok * 4), G.Guarded(n_tok)
+    mask = G.dev(pk.mask)
+    ndev = None
+    if n_on_device:
+        ndev = torch.zeros(1, dtype=torch.int64, device="cuda")
+        api.hilore_mask_count(mask, n_tok, ndev)
+    api.hilore_grpo_coeffs_packed(G.dev(ro.rewards), ro.n_resp, ro.G, resp_offset, n_seq, dev_i32(pk.cu_seqlens), n_tok,
+                                  G.dev(pk.logp_new), G.dev(pk.logp_old), G.dev(pk.logp_ref) if beta else None, mask,
+                                  0 if n_on_device else (ro.n_valid if N is None else N), ndev, 0.2, beta, 1e-6, adv.ptr(),
+                                  omega.ptr(), ratio.ptr(), chi.ptr())
+    return (adv.numpy(np.float32, (n_seq,)), omega.numpy(np.float32, (n_tok,)), ratio.numpy(np.float32, (n_tok,)),
+            chi.numpy(np.uint8, (n_tok,)))
+
+
+def check(ro, pk, got, beta, N):
+    adv, omega, ratio, chi = got
+    adv_o = oracle.group_advantages(ro.rewards, ro.G)[pk.rows]
+    w, r, c = oracle.grpo_coeffs_packed(adv_o, pk.cu_seqlens, pk.logp_new, pk.logp_old, pk.logp_ref if beta else None,
+                                        pk.mask, N_norm=N, beta=beta)
+    lens = np.diff(pk.cu_seqlens)
+    assert G.rel_err(adv, adv_o).max(initial=0) <= RTOL and np.array_equal(adv == 0, adv_o == 0)
+    hi, lo = np.float32(1.2), np.float32(0.8)
+    near = (np.abs(r - hi) <= 4 * np.spacing(hi)) | (np.abs(r - lo) <= 4 * np.spacing(lo))
+    assert not np.any((chi != c) & ~near)
+    assert G.rel_err(ratio, r).max(initial=0) <= RTOL
+    ok = ~near
+    err = G.rel_err(omega[ok], w[ok])
+    kl = beta * pk.mask / N * (1 - np.exp(pk.logp_ref.astype(np.float64) - pk.logp_new))
+    floor = RTOL * np.maximum(np.abs(w.astype(np.float64) - kl), np.abs(kl))[ok]
+    assert np.all((err <= RTOL) | (np.abs(omega[ok].astype(np.float64) - w[ok]) <= floor))
+    assert np.all(omega[pk.mask == 0] == 0)
+    return lens
+
+
+@pytest.mark.parametrize("beta", [0.0, 1e-3])
+@pytest.mark.parametrize("P,G_,T,max_prompt", [(8, 8, 700, 300), (3, 4, 36, 5), (64, 16, 64, 3)])
+def test_packed_coeffs_match_oracle(P, G_, T, max_prompt, beta):
+    ro = synth.rollout(31, P, G_, T, lengths="uniform", min_len=1, rewards="bernoulli", equal_group_fraction=0.25)
+    ro.logp_old[:] = ro.logp_new + np.random.default_rng(4).normal(0, 0.12, ro.logp_new.shape).astype(np.float32)
+    pk = synth.pack_rollout(ro, 6, max_prompt=max_prompt)
+    got = packed_gpu(ro, pk, beta=beta)
+    check(ro, pk, got, beta, ro.n_valid)
+    # the same tokens through the dense kernel: identical bits (same arithmetic per token)
+    dense = G.grpo_coeffs(ro, N_norm=ro.n_valid, beta=beta)
+    seq = np.repeat(np.arange(len(pk.rows)), np.diff(pk.cu_seqlens))
+    resp = pk.dense_t >= 0
+    i, t = pk.rows[seq[resp]], pk.dense_t[resp]
+    assert np.array_equal(got[1][resp], dense["omega"][i, t])
+    assert np.array_equal(got[2][resp], dense["ratio"][i, t])
+
+
+def test_packed_microbatch_slice_device_normaliser_and_empty_sequences():
+    ro = synth.rollout(32, 4, 8, 128, lengths="uniform", min_len=2)
+    rows = np.arange(8, 24)                                  # a microbatch: responses 8..23 of the rollout batch
+    pk = synth.pack_rollout(ro, 2, rows=rows, max_prompt=17)
+    # insert empty sequences by repeating boundaries: sequences 3 and 9 own nothing
+    lens = np.diff(pk.cu_seqlens).astype(np.int64)
+    keep = np.ones(len(rows), bool)
+    keep[[3, 9]] = False
+    cu2 = np.zeros(len(rows) + 1, np.int64)
+    np.cumsum(np.where(keep, lens, 0), out=cu2[1:])
+    sel = np.concatenate([np.arange(pk.cu_seqlens[j], pk.cu_seqlens[j + 1]) for j in range(len(rows)) if keep[j]])
+    pk2 = synth.PackedRollout(cu2.astype(np.int32), rows, pk.logp_new[sel].copy(), pk.logp_old[sel].copy(),
+                              pk.logp_ref[sel].copy(), pk.mask[sel].copy(), pk.dense_t[sel].copy())
+    N = int(pk2.mask.sum())
+    got = packed_gpu(ro, pk2, beta=1e-3, resp_offset=8, n_on_device=True)
+    check(ro, pk2, got, 1e-3, N)
+
+
+def test_packed_argument_errors():
+    z = torch.zeros(16, device="cuda")
+    zi = torch.zeros(4, dtype=torch.int32, device="cuda")
+    m = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    call = lambda **kw: api.hilore_grpo_coeffs_packed(
+        kw.get("rewards", z), kw.get("n_resp", 8), kw.get("G", 4), kw.get("off", 0), kw.get("n_seq", 3), kw.get("cu", zi),
+        kw.get("n_tok", 16), z, z, kw.get("ref", None), m, kw.get("N", 5), None, 0.2, kw.get("beta", 0.0), 1e-6,
+        kw.get("adv", z), z, None, None, check=False)
+    assert call() == api.OK
+    assert call(adv=None) == api.INVALID_ARG
+    assert call(cu=None) == api.INVALID_ARG
+    assert call(N=0) == api.ZERO_NORM
+    assert call(beta=0.1) == api.INVALID_ARG
+    assert call(off=6) == api.SHAPE
+    assert call(n_resp=7) == api.SHAPE
+    assert call(n_tok=1 << 31) == api.SHAPE
+    assert call(n_seq=0, n_tok=0) == api.OK
+
+
+@pytest.mark.parametrize("row_shift", [0, 1])
+@pytest.mark.parametrize("min_prompt", [0, 1])
+def test_packed_exposure_matches_oracle(row_shift, min_prompt):
+    ro = synth.rollout(33, 6, 4, 300, lengths="uniform", min_len=1)
+    pk = synth.pack_rollout(ro, 8, max_prompt=40, min_prompt=min_prompt)
+    n_tok, n_seq, U = pk.n_tok, len(pk.rows), 11
+    rng = np.random.default_rng(3)
+    omega = (rng.standard_normal(n_tok).astype(np.float32) * 1e-4 * pk.mask).astype(np.float32)
+    ld = n_tok + 5
+    rms = rng.random((U, ld), dtype=np.float32) + np.float32(0.1)
+    nws = api.hilore_workspace_bytes(U, n_tok)
+    ws, E, sw = G.Guarded(nws), G.Guarded(U * 4), G.Guarded(4)
+    api.hilore_unit_exposure_packed(G.dev(omega), G.dev(pk.mask), n_tok, dev_i32(pk.cu_seqlens), n_seq, G.dev(rms), U, ld,
+                                    row_shift, 1e-8, E.ptr(), sw.ptr(), ws.ptr(), nws)
+    ws.numpy(np.uint8, (nws,))
+    oE, osw = oracle.unit_exposure_packed(omega, pk.mask, pk.cu_seqlens, rms, row_shift=row_shift)
+    assert G.rel_err(E.numpy(np.float32, (U,)), oE).max() <= RTOL
+    assert abs(float(sw.numpy(np.float32, (1,))[0]) - osw) <= RTOL * osw
