@@ -294,6 +294,14 @@ double hilore_risk_budget(double delta, int64_t N_b, int64_t N_total);
 int hilore_relative_error(const void *x, const void *xhat, int64_t rows, int64_t cols, int64_t ld, int64_t ld_hat,
                           double *e_out, double *norms2, void *workspace, size_t workspace_bytes, void *stream);
 size_t hilore_relative_error_workspace_bytes(void);
+/*
+ * The same e^L for x_hat = recover(compress(x)) in format fmt, fused: x is read once (2 B per element), encoded
+ * and decoded in registers with the routines of hilore_compress / hilore_recover (x_hat is bit for bit what
+ * they would produce), nothing else is written.  Shape and alignment rules of hilore_compress; workspace,
+ * outputs and determinism as hilore_relative_error.  A unit with NaN codes gives e^L = NaN.
+ */
+int hilore_codec_relative_error(const void *x, int64_t rows, int64_t cols, int64_t ld, int32_t fmt, int32_t block,
+                                double *e_out, double *norms2, void *workspace, size_t workspace_bytes, void *stream);
 double hilore_fit_kappa(const double *x, const double *y, int64_t n);
 
 /* One recovery unit of a microbatch: where its bf16 bundle lives and where its L representation goes.

@@ -3,6 +3,7 @@
 // the norms) and the closed-form susceptibility fit (Eq. "susceptibility").  Used at initialisation on the
 // calibration microbatches, not in the per-microbatch hot loop.
 #include "common.cuh"
+#include "codec.cuh"
 
 namespace hilore {
 
@@ -82,9 +83,103 @@ __global__ void __launch_bounds__(32) relerr_final_kernel(const double *partial,
     }
 }
 
+// e^L of format FMT on x without materialising codes or x_hat: each thread encodes its two 16-element chunks with
+// the compress kernel's own routine, decodes them with the recover kernel's own routine (so x_hat is bit for
+// bit what hilore_recover would write) and accumulates both norms.  x is read once: 2 B per element.
+template <int FMT>
+__global__ void __launch_bounds__(kCodecThreads) codec_relerr_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t cols,
+                                                                    int64_t ld, double *__restrict__ partial)
+{
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int64_t cpr = cols >> 4, n = rows * cpr; // chunks; a multiple of 4 (cols % 64 == 0)
+    const int64_t steps = (n + 2 * kCodecThreads - 1) / (2 * kCodecThreads);
+    const int64_t s_begin = (steps / gridDim.x) * blockIdx.x + ((steps % gridDim.x) * blockIdx.x) / gridDim.x;
+    const int64_t s_end = (steps / gridDim.x) * (blockIdx.x + 1) + ((steps % gridDim.x) * (blockIdx.x + 1)) / gridDim.x;
+    double err = 0.0, nrm = 0.0;
+    for (int64_t st = s_begin; st < s_end; ++st) { // the trip count is uniform over the CTA (shuffles inside)
+        const int64_t ca = st * 2 * kCodecThreads + tid, cb = ca + kCodecThreads;
+        uint32_t wa[8], wb[8];
+        zero8(wa); // a chunk past the end reads as zeros: code 0, x_hat 0, no contribution
+        zero8(wb);
+        if (ca < n) {
+            const int64_t r = ca / cpr;
+            ld_global_256(x + r * ld + (ca - r * cpr) * 16, wa);
+        }
+        if (cb < n) {
+            const int64_t r = cb / cpr;
+            ld_global_256(x + r * ld + (cb - r * cpr) * 16, wb);
+        }
+        uint4 qa, qb;
+        float s, unused;
+        process_pair<FMT, true, false>(wa, wb, lane, qa, qb, s, unused);
+        float sa = 1.0f, sb = 1.0f;
+        if (FMT != HILORE_FMT_E4M3FN_RAW) { // the scale of chunk a's block sits in lane 0 of the quad, of chunk b's in lane 2
+            sa = __shfl_sync(0xFFFFFFFFu, s, (lane & 28));
+            sb = __shfl_sync(0xFFFFFFFFu, s, (lane & 28) | 2);
+        }
+        uint32_t oa[8], ob[8];
+        decode16<FMT>(qa, sa, oa);
+        decode16<FMT>(qb, sb, ob);
+        float e0, m0, e1, m1;
+        err16(wa, oa, e0, m0);
+        err16(wb, ob, e1, m1);
+        err += (double)e0 + (double)e1;
+        nrm += (double)m0 + (double)m1;
+    }
+    __shared__ double sm[kCodecThreads / 32][2];
+    err = warp_sum(err);
+    nrm = warp_sum(nrm);
+    if (lane == 0) {
+        sm[tid >> 5][0] = err;
+        sm[tid >> 5][1] = nrm;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double e = 0.0, m = 0.0;
+        for (int w = 0; w < kCodecThreads / 32; ++w) {
+            e += sm[w][0];
+            m += sm[w][1];
+        }
+        partial[2 * blockIdx.x] = e;
+        partial[2 * blockIdx.x + 1] = m;
+    }
+}
+
 } // namespace hilore
 
 using namespace hilore;
+
+extern "C" int hilore_codec_relative_error(const void *x, int64_t rows, int64_t cols, int64_t ld, int32_t fmt, int32_t block,
+                                           double *e_out, double *norms2, void *workspace, size_t workspace_bytes,
+                                           void *stream)
+{
+    if (rows < 0 || cols <= 0 || !e_out || !workspace || (rows > 0 && !x))
+        return HILORE_INVALID_ARG;
+    if (fmt != HILORE_FMT_E4M3FN_RAW && fmt != HILORE_FMT_E4M3FN_BLK && fmt != HILORE_FMT_INT8_BLK)
+        return HILORE_INVALID_ARG;
+    if (cols % 64 != 0 || ld < cols || (fmt == HILORE_FMT_E4M3FN_RAW ? block != 0 : block != 64))
+        return HILORE_SHAPE;
+    if (ld % 16 != 0 || !aligned(x, 32) || !aligned(e_out, 8) || !aligned(norms2, 8) || !aligned(workspace, 16))
+        return HILORE_ALIGN;
+    if (workspace_bytes < hilore_relative_error_workspace_bytes())
+        return HILORE_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t steps = (rows * (cols / 16) + 2 * kCodecThreads - 1) / (2 * kCodecThreads);
+    int64_t grid = (int64_t)sm_count() * 4;
+    if (grid > kErrMaxGrid) grid = kErrMaxGrid;
+    if (grid > steps) grid = steps;
+    if (grid < 1) grid = 1;
+    double *partial = static_cast<double *>(workspace);
+    const uint16_t *xp = static_cast<const uint16_t *>(x);
+    if (fmt == HILORE_FMT_E4M3FN_RAW)
+        codec_relerr_kernel<HILORE_FMT_E4M3FN_RAW><<<(unsigned)grid, kCodecThreads, 0, st>>>(xp, rows, cols, ld, partial);
+    else if (fmt == HILORE_FMT_E4M3FN_BLK)
+        codec_relerr_kernel<HILORE_FMT_E4M3FN_BLK><<<(unsigned)grid, kCodecThreads, 0, st>>>(xp, rows, cols, ld, partial);
+    else
+        codec_relerr_kernel<HILORE_FMT_INT8_BLK><<<(unsigned)grid, kCodecThreads, 0, st>>>(xp, rows, cols, ld, partial);
+    relerr_final_kernel<<<1, 32, 0, st>>>(partial, (int)grid, e_out, norms2);
+    return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+}
 
 extern "C" size_t hilore_relative_error_workspace_bytes(void) { return (size_t)kErrMaxGrid * 2 * sizeof(double); }
 

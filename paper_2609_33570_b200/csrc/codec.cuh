@@ -179,7 +179,7 @@ template <int FMT> __device__ __noinline__ uint4 encode16_careful(uint4 lo, uint
 }
 
 // max |bits| over the finite elements only (rare path, by value)
-__device__ __noinline__ uint32_t absmax16_finite(uint4 lo, uint4 hi)
+static __device__ __noinline__ uint32_t absmax16_finite(uint4 lo, uint4 hi)
 {
     const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
     uint32_t m = 0;

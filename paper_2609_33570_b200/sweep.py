@@ -73,6 +73,24 @@ def coeffs_point(log2_slots, reps, G=16, T=1024):
             "gbs": 13 * slots / t / 1e6}
 
 
+def relerr_point(rows, cols, fmt, reps):
+    """e^L of one unit: fused (x read once, codec in registers) against compress + recover + compare."""
+    block = 0 if fmt == api.FMT_E4M3FN_RAW else 64
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4)
+    pool = max(1, min(8, -(-3 * L2_BYTES // (rows * cols * 2))))
+    base = synth.activation_unit_device(gen, min(rows, 4096), cols)
+    xs = [base.repeat(-(-rows // base.shape[0]), 1)[:rows].contiguous() for _ in range(pool)]
+    nws = api.hilore_relative_error_workspace_bytes()
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    e = torch.zeros(1, dtype=torch.float64, device="cuda")
+    fused = [lambda i=i: api.hilore_codec_relative_error(xs[i], rows, cols, cols, fmt, block, e, None, ws, nws)
+             for i in range(pool)]
+    t = _time(fused, reps)
+    return {"kernel": "codec_relative_error", "rows": rows, "cols": cols, "fmt": fmt, "us": t * 1e3,
+            "gbs": 2 * rows * cols / t / 1e6, "e": e.item()}
+
+
 def coeffs_packed_point(log2_tokens, reps, G=8, mean_len=2048):
     """The coefficient kernel on the packed layout: sequences of U{mean_len/2 .. 3 mean_len/2} tokens back to back."""
     import numpy as np
@@ -174,6 +192,8 @@ def main():
     if not a.no_coeffs:
         for ls in range(16, 25):
             print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
+        for fmt in a.fmts:
+            print(json.dumps(relerr_point(65536, 8960, fmt, a.reps)), flush=True)
         for ls in (15, 20, 24, 27):
             print(json.dumps(coeffs_packed_point(ls, a.reps)), flush=True)
         for ls in (20, 24, 27):
