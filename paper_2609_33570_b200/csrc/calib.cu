@@ -111,7 +111,8 @@ __global__ void __launch_bounds__(kCodecThreads) codec_relerr_kernel(const uint1
         }
         uint4 qa, qb;
         float s, unused;
-        process_pair<FMT, true, false>(wa, wb, lane, qa, qb, s, unused);
+        bool careful_unused;
+        process_pair<FMT, true, false>(wa, wb, lane, qa, qb, s, unused, careful_unused);
         float sa = 1.0f, sb = 1.0f;
         if (FMT != HILORE_FMT_E4M3FN_RAW) { // the scale of chunk a's block sits in lane 0 of the quad, of chunk b's in lane 2
             sa = __shfl_sync(0xFFFFFFFFu, s, (lane & 28));

@@ -165,7 +165,7 @@ template <int FMT> __device__ __forceinline__ uint32_t encode1_careful(uint32_t 
 }
 
 // Rare path, kept out of line and fed by value so that the common path keeps its data in registers.
-template <int FMT> __device__ __noinline__ uint4 encode16_careful(uint4 lo, uint4 hi, float inv)
+template <int FMT> __device__ __forceinline__ uint4 encode16_careful_inl(uint4 lo, uint4 hi, float inv)
 {
     const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
     uint32_t c[4];
@@ -178,8 +178,13 @@ template <int FMT> __device__ __noinline__ uint4 encode16_careful(uint4 lo, uint
     return make_uint4(c[0], c[1], c[2], c[3]);
 }
 
+template <int FMT> __device__ __noinline__ uint4 encode16_careful(uint4 lo, uint4 hi, float inv)
+{
+    return encode16_careful_inl<FMT>(lo, hi, inv);
+}
+
 // max |bits| over the finite elements only (rare path, by value)
-static __device__ __noinline__ uint32_t absmax16_finite(uint4 lo, uint4 hi)
+__device__ __forceinline__ uint32_t absmax16_finite_inl(uint4 lo, uint4 hi)
 {
     const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
     uint32_t m = 0;
@@ -192,6 +197,8 @@ static __device__ __noinline__ uint32_t absmax16_finite(uint4 lo, uint4 hi)
     return m;
 }
 
+static __device__ __noinline__ uint32_t absmax16_finite(uint4 lo, uint4 hi) { return absmax16_finite_inl(lo, hi); }
+
 #define HILORE_LO4(w) make_uint4((w)[0], (w)[1], (w)[2], (w)[3])
 #define HILORE_HI4(w) make_uint4((w)[4], (w)[5], (w)[6], (w)[7])
 
@@ -202,26 +209,31 @@ __device__ __forceinline__ void chunk_pass(const uint32_t (&w)[8], float inv, ui
 {
     const uint64_t inv2 = f32x2_pack(inv, inv);
     uint64_t acc = 0; // {0.0f, 0.0f}
-    uint32_t h[8];    // two codes per word
+    uint32_t cw[4];   // four codes per word
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        uint64_t x = f32x2_pack(bf16_lo(w[i]), bf16_hi(w[i]));
-        if (SUMS)
-            acc = f32x2_fma(x, x, acc);
+    for (int i = 0; i < 4; ++i) {
+        uint64_t xa = f32x2_pack(bf16_lo(w[2 * i]), bf16_hi(w[2 * i]));
+        uint64_t xb = f32x2_pack(bf16_lo(w[2 * i + 1]), bf16_hi(w[2 * i + 1]));
+        if (SUMS) {
+            acc = f32x2_fma(xa, xa, acc);
+            acc = f32x2_fma(xb, xb, acc);
+        }
         if (CODES) {
-            if (FMT != HILORE_FMT_E4M3FN_RAW)
-                x = f32x2_mul(x, inv2); // fl32(x * inv), each lane rounded to nearest even
-            float lo, hi;
-            f32x2_unpack(x, lo, hi);
+            if (FMT != HILORE_FMT_E4M3FN_RAW) { // fl32(x * inv), each lane rounded to nearest even
+                xa = f32x2_mul(xa, inv2);
+                xb = f32x2_mul(xb, inv2);
+            }
+            float a0, a1, b0, b1;
+            f32x2_unpack(xa, a0, a1);
+            f32x2_unpack(xb, b0, b1);
             if (FMT == HILORE_FMT_INT8_BLK)
-                h[i] = int8_code(lo) | (int8_code(hi) << 8);
+                cw[i] = int8_code(a0) | (int8_code(a1) << 8) | (int8_code(b0) << 16) | (int8_code(b1) << 24);
             else
-                h[i] = cvt_e4m3x2(hi, lo);
+                cw[i] = cvt_e4m3x4(a0, a1, b0, b1);
         }
     }
     if (CODES)
-        codes = make_uint4(__byte_perm(h[0], h[1], 0x5410), __byte_perm(h[2], h[3], 0x5410),
-                           __byte_perm(h[4], h[5], 0x5410), __byte_perm(h[6], h[7], 0x5410));
+        codes = make_uint4(cw[0], cw[1], cw[2], cw[3]);
     if (SUMS) {
         float lo, hi;
         f32x2_unpack(acc, lo, hi);
@@ -236,9 +248,12 @@ __device__ __forceinline__ void chunk_pass(const uint32_t (&w)[8], float inv, ui
 //          division per thread instead of four.  `s_store` is the scale of chunk 0's block in lanes with
 //          (lane & 3) == 0 and of chunk 1's block in lanes with (lane & 3) == 2.
 //   SUMS:  `bsum` is the block sum of squares of chunk 0's block in even lanes, of chunk 1's in odd lanes.
-template <int FMT, bool CODES, bool SUMS>
+//   LATER: blocks that need the careful rules (Inf, NaN, overflow of the unscaled cast) are only reported in
+//          `careful`; their codes and scales come out wrong here and the caller repairs them with
+//          careful_pair_fixup after its stores.  This keeps calls and their register traffic out of the loop.
+template <int FMT, bool CODES, bool SUMS, bool LATER = false>
 __device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint32_t (&w1)[8], int lane, uint4 &c0,
-                                             uint4 &c1, float &s_store, float &bsum)
+                                             uint4 &c1, float &s_store, float &bsum, bool &careful)
 {
     constexpr float Q = QMax<FMT>::value;
     float inv0 = 1.0f, inv1 = 1.0f;
@@ -256,7 +271,7 @@ __device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint
             m0 = mp & 0xFFFFu;
             m1 = mp >> 16;
             careful0 = careful1 = (m0 >= 0x7F80u) || (m1 >= 0x7F80u); // uniform over the quad
-            if (careful0) { // Inf or NaN in one of the two blocks: absmax over the finite elements only
+            if (!LATER && careful0) { // Inf or NaN in one of the two blocks: absmax over the finite elements only
                 const uint32_t quad_mask = 0xFu << (lane & 28);
                 uint32_t f0 = absmax16_finite(HILORE_LO4(w0), HILORE_HI4(w0));
                 uint32_t f1 = absmax16_finite(HILORE_LO4(w1), HILORE_HI4(w1));
@@ -279,10 +294,12 @@ __device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint
     float ss0 = 0.0f, ss1 = 0.0f;
     chunk_pass<FMT, CODES, SUMS>(w0, inv0, c0, ss0);
     chunk_pass<FMT, CODES, SUMS>(w1, inv1, c1, ss1);
-    if (CODES) {
+    if (CODES && !LATER) {
         if (careful0) c0 = encode16_careful<FMT>(HILORE_LO4(w0), HILORE_HI4(w0), inv0);
         if (careful1) c1 = encode16_careful<FMT>(HILORE_LO4(w1), HILORE_HI4(w1), inv1);
     }
+    if (CODES && LATER)
+        careful = careful0 || careful1;
     if (SUMS) { // quad reduction of both blocks' sums with two shuffles
         const bool odd = lane & 1;
         float keep = odd ? ss1 : ss0;
@@ -296,6 +313,42 @@ __device__ __forceinline__ void zero8(uint32_t (&w)[8])
 {
 #pragma unroll
     for (int i = 0; i < 8; ++i) w[i] = 0;
+}
+
+// Redo the two chunks of a thread with the full rule set and overwrite what the fast path stored for them.
+// Rare (a block holds Inf or NaN; the unscaled cast meets a magnitude above 464), so it re-reads the chunks
+// instead of keeping them alive.  For the block formats the condition is uniform over a quad and all four lanes
+// come here together; xa / xb is nullptr where the thread has no chunk.  The scale slots are written by the
+// same lanes as on the fast path (lane 0 of the quad for chunk a's block, lane 2 for chunk b's).
+template <int FMT>
+__device__ __forceinline__ void careful_pair_fixup(const uint16_t *xa, const uint16_t *xb, uint8_t *ca, uint8_t *cb, float *sa,
+                                                float *sb, int lane)
+{
+    constexpr float Q = QMax<FMT>::value;
+    uint32_t w0[8], w1[8];
+    if (xa) ld_global_256(xa, w0);
+    else zero8(w0);
+    if (xb) ld_global_256(xb, w1);
+    else zero8(w1);
+    float inv0 = 1.0f, inv1 = 1.0f;
+    if (FMT != HILORE_FMT_E4M3FN_RAW) {
+        const uint32_t quad_mask = 0xFu << (lane & 28);
+        uint32_t f0 = absmax16_finite_inl(HILORE_LO4(w0), HILORE_HI4(w0));
+        uint32_t f1 = absmax16_finite_inl(HILORE_LO4(w1), HILORE_HI4(w1));
+        f0 = max(f0, __shfl_xor_sync(quad_mask, f0, 1));
+        f1 = max(f1, __shfl_xor_sync(quad_mask, f1, 1));
+        f0 = max(f0, __shfl_xor_sync(quad_mask, f0, 2));
+        f1 = max(f1, __shfl_xor_sync(quad_mask, f1, 2));
+        const float a0 = __uint_as_float(f0 << 16), a1 = __uint_as_float(f1 << 16);
+        const bool unit0 = f0 <= UnitScaleBelow<FMT>::value, unit1 = f1 <= UnitScaleBelow<FMT>::value;
+        inv0 = unit0 ? 1.0f : __fdiv_rn(Q, a0);
+        inv1 = unit1 ? 1.0f : __fdiv_rn(Q, a1);
+        const int q = lane & 3;
+        if (q == 0 && xa) *sa = unit0 ? 1.0f : __fdiv_rn(a0, Q);
+        if (q == 2 && xb) *sb = unit1 ? 1.0f : __fdiv_rn(a1, Q);
+    }
+    if (xa) *reinterpret_cast<uint4 *>(ca) = encode16_careful_inl<FMT>(HILORE_LO4(w0), HILORE_HI4(w0), inv0);
+    if (xb) *reinterpret_cast<uint4 *>(cb) = encode16_careful_inl<FMT>(HILORE_LO4(w1), HILORE_HI4(w1), inv1);
 }
 
 // Compress (CODES) and / or collect the token RMS (SUMS) of rows [r0, r1) of one unit.
@@ -340,7 +393,8 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
                 ld_global_256(xp + kCodecThreads * 16, wb);
                 uint4 qa, qb;
                 float s, ss;
-                process_pair<FMT, CODES, SUMS>(wa, wb, lane, qa, qb, s, ss);
+                bool careful = false;
+                process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful);
                 if (CODES) {
                     *reinterpret_cast<uint4 *>(cp) = qa;
                     *reinterpret_cast<uint4 *>(cp + kCodecThreads * 16) = qb;
@@ -348,6 +402,9 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
                         if (q == 0) sp[0] = s;
                         if (q == 2) sp[kCodecThreads / 4] = s;
                     }
+                    if (careful)
+                        careful_pair_fixup<FMT>(xp, xp + kCodecThreads * 16, cp, cp + kCodecThreads * 16, sp,
+                                                sp + kCodecThreads / 4, lane);
                 }
                 if (SUMS) {
                     if (q == 0) bp[0] = ss;
@@ -365,17 +422,21 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
             uint32_t wa[8], wb[8];
             zero8(wa);
             zero8(wb);
+            const uint16_t *xa_ptr = nullptr, *xb_ptr = nullptr;
             if (va) {
                 const uint32_t r = __umulhi(ca, magic);
-                ld_global_256(xb + (int64_t)r * ld + (int64_t)(ca - r * cpr) * 16, wa);
+                xa_ptr = xb + (int64_t)r * ld + (int64_t)(ca - r * cpr) * 16;
+                ld_global_256(xa_ptr, wa);
             }
             if (vb) {
                 const uint32_t r = __umulhi(cb, magic);
-                ld_global_256(xb + (int64_t)r * ld + (int64_t)(cb - r * cpr) * 16, wb);
+                xb_ptr = xb + (int64_t)r * ld + (int64_t)(cb - r * cpr) * 16;
+                ld_global_256(xb_ptr, wb);
             }
             uint4 qa, qb;
             float s, ss;
-            process_pair<FMT, CODES, SUMS>(wa, wb, lane, qa, qb, s, ss);
+            bool careful = false;
+            process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful);
             if (CODES) {
                 if (va) *reinterpret_cast<uint4 *>(cb_ + (size_t)ca * 16) = qa;
                 if (vb) *reinterpret_cast<uint4 *>(cb_ + (size_t)cb * 16) = qb;
@@ -383,6 +444,9 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
                     if (q == 0 && va) sb[ca >> 2] = s;
                     if (q == 2 && vb) sb[cb >> 2] = s;
                 }
+                if (careful)
+                    careful_pair_fixup<FMT>(va ? xa_ptr : nullptr, vb ? xb_ptr : nullptr, cb_ + (size_t)ca * 16,
+                                            cb_ + (size_t)cb * 16, sb + (ca >> 2), sb + (cb >> 2), lane);
             }
             if (SUMS) {
                 if (q == 0 && va) sm_blocksum[ca >> 2] = ss;

@@ -57,6 +57,20 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo)
     return r;
 }
 
+// Four fp32 -> four E4M3FN codes in one word, x0 in the lowest byte.  The two 16-bit halves are joined inside
+// the asm block, so no zero-extension of the halves is emitted.
+__device__ __forceinline__ uint32_t cvt_e4m3x4(float x0, float x1, float x2, float x3)
+{
+    uint32_t r;
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 lo, %2, %1;\n\t"
+        "cvt.rn.satfinite.e4m3x2.f32 hi, %4, %3;\n\t"
+        "mov.b32 %0, {lo, hi};\n\t}"
+        : "=r"(r)
+        : "f"(x0), "f"(x1), "f"(x2), "f"(x3));
+    return r;
+}
+
 // Two E4M3FN codes (low 16 bits of `c`) -> two fp16 (exact), packed.
 __device__ __forceinline__ uint32_t cvt_e4m3x2_to_f16x2(uint32_t c)
 {
