@@ -9,15 +9,16 @@ namespace hilore {
 
 // Compress / token-RMS pass over rows [r0, r1) of one unit, specialised on what the unit asks for.
 template <int FMT>
-__device__ __forceinline__ void compress_unit(const hilore_unit &u, int op, int64_t r0, int64_t r1, float *sm, int pf)
+__device__ __forceinline__ void compress_unit(const hilore_unit &u, int op, int64_t r0, int64_t r1, float *sm, int pf,
+                                              const uint32_t *tab)
 {
     const uint16_t *x = static_cast<const uint16_t *>(u.x);
     if (op == OP_STATS)
-        compress_rows<HILORE_FMT_E4M3FN_RAW, false, true>(x, nullptr, nullptr, u.row_rms, u.cols, u.ld, r0, r1, sm, pf);
+        compress_rows<HILORE_FMT_E4M3FN_RAW, false, true>(x, nullptr, nullptr, u.row_rms, u.cols, u.ld, r0, r1, sm, pf, tab);
     else if (u.row_rms != nullptr)
-        compress_rows<FMT, true, true>(x, u.codes, u.scales, u.row_rms, u.cols, u.ld, r0, r1, sm, pf);
+        compress_rows<FMT, true, true>(x, u.codes, u.scales, u.row_rms, u.cols, u.ld, r0, r1, sm, pf, tab);
     else
-        compress_rows<FMT, true, false>(x, u.codes, u.scales, nullptr, u.cols, u.ld, r0, r1, sm, pf);
+        compress_rows<FMT, true, false>(x, u.codes, u.scales, nullptr, u.cols, u.ld, r0, r1, sm, pf, tab);
 }
 
 // FMT >= 0: every unit of the launch has this format (the common case; the hot loop is compiled for it).
@@ -25,15 +26,19 @@ __device__ __forceinline__ void compress_unit(const hilore_unit &u, int op, int6
 template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_kernel(const __grid_constant__ CodecWork wk)
 {
     __shared__ float sm_blocksum[kBlockSumSlots];
+    __shared__ uint32_t sm_tab[2][kScaleTableWords]; // scale tables: [0] Q = 448, [1] Q = 127
+    if (FMT < 0 || FMT == HILORE_FMT_E4M3FN_BLK) fill_scale_table<HILORE_FMT_E4M3FN_BLK>(sm_tab[0]);
+    if (FMT < 0 || FMT == HILORE_FMT_INT8_BLK) fill_scale_table<HILORE_FMT_INT8_BLK>(sm_tab[1]);
+    __syncthreads();
     JobCursor cur;
     Job j;
     while (next_job(wk, cur, j)) {
         if (j.op == OP_RECOVER)
             continue;
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
-        if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch);
-        else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch);
-        else compress_unit<HILORE_FMT_INT8_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch);
+        if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
+        else compress_unit<HILORE_FMT_INT8_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[1]);
     }
 }
 

@@ -105,6 +105,31 @@ template <int FMT> struct UnitScaleBelow {
     static constexpr uint32_t value = (FMT == HILORE_FMT_INT8_BLK) ? 0x02FEu : 0x03E0u;
 };
 
+// Smallest |bf16| pattern for which both s = amax / Q and inv = Q / amax are normal fp32 numbers
+// (Q = 448: amax >= 1.75 * 2^-118; Q = 127: amax >= 1.984375 * 2^-120).  From here up to the largest finite
+// pattern the two quotients follow from the 7 mantissa bits alone (scale table below).
+template <int FMT> struct TableScaleFrom {
+    static constexpr uint32_t value = (FMT == HILORE_FMT_INT8_BLK) ? 0x03FEu : 0x04E0u;
+};
+
+// Scale table.  amax is a bf16 number v * 2^E with v = 1 + m / 128, so fl32(amax / Q) = fl32(v / Q) * 2^E and
+// fl32(Q / amax) = fl32(Q / v) * 2^-E exactly while the results stay normal: the correctly rounded quotient
+// depends on m only, and the power of two is an integer addition to the exponent field.  Entry m holds the
+// bit patterns of fl32(v / Q) and fl32(Q / v) with the exponent bias folded in, so that
+//     bits(s) = tab[m] + (amax_bits & 0x7F80) * 65536,    bits(inv) = tab[128 + m] - (amax_bits & 0x7F80) * 65536.
+// Two IEEE divisions per block become one shared-memory load and one integer multiply-add per lane.
+constexpr int kScaleTableWords = 256; // per format family: [0,128) for s, [128,256) for inv
+
+template <int FMT> __device__ __forceinline__ void fill_scale_table(uint32_t *tab)
+{
+    constexpr float Q = QMax<FMT>::value;
+    for (int i = threadIdx.x; i < 128; i += blockDim.x) {
+        const float v = 1.0f + (float)i * 0.0078125f;
+        tab[i] = __float_as_uint(__fdiv_rn(v, Q)) - (127u << 23);
+        tab[128 + i] = __float_as_uint(__fdiv_rn(Q, v)) + (127u << 23);
+    }
+}
+
 __device__ __forceinline__ uint32_t int8_code(float q)
 {
     int v = __float2int_rn(q);
@@ -251,9 +276,12 @@ __device__ __forceinline__ void chunk_pass(const uint32_t (&w)[8], float inv, ui
 //   LATER: blocks that need the careful rules (Inf, NaN, overflow of the unscaled cast) are only reported in
 //          `careful`; their codes and scales come out wrong here and the caller repairs them with
 //          careful_pair_fixup after its stores.  This keeps calls and their register traffic out of the loop.
+//   `tab` (LATER only): the scale table of this format in shared memory; blocks whose amax lies outside the
+//          table's range and is not a unit-scale block are reported as careful too.
 template <int FMT, bool CODES, bool SUMS, bool LATER = false>
 __device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint32_t (&w1)[8], int lane, uint4 &c0,
-                                             uint4 &c1, float &s_store, float &bsum, bool &careful)
+                                             uint4 &c1, float &s_store, float &bsum, bool &careful,
+                                             const uint32_t *tab = nullptr)
 {
     constexpr float Q = QMax<FMT>::value;
     float inv0 = 1.0f, inv1 = 1.0f;
@@ -270,7 +298,7 @@ __device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint
             mp = maxnan_bf16x2(mp, __shfl_xor_sync(0xFFFFFFFFu, mp, 2));
             m0 = mp & 0xFFFFu;
             m1 = mp >> 16;
-            careful0 = careful1 = (m0 >= 0x7F80u) || (m1 >= 0x7F80u); // uniform over the quad
+            if (!LATER) careful0 = careful1 = (m0 >= 0x7F80u) || (m1 >= 0x7F80u); // uniform over the quad
             if (!LATER && careful0) { // Inf or NaN in one of the two blocks: absmax over the finite elements only
                 const uint32_t quad_mask = 0xFu << (lane & 28);
                 uint32_t f0 = absmax16_finite(HILORE_LO4(w0), HILORE_HI4(w0));
@@ -281,9 +309,18 @@ __device__ __forceinline__ void process_pair(const uint32_t (&w0)[8], const uint
                 m1 = max(f1, __shfl_xor_sync(quad_mask, f1, 2));
             }
             const int q = lane & 3;
-            const float a = __uint_as_float(((q & 2) ? m1 : m0) << 16);
-            const float r = __fdiv_rn((q & 1) ? Q : a, (q & 1) ? a : Q); // s in even lanes, inv in odd lanes
             const bool unit0 = m0 <= UnitScaleBelow<FMT>::value, unit1 = m1 <= UnitScaleBelow<FMT>::value;
+            float r; // s in even lanes, inv in odd lanes
+            if (LATER) {
+                constexpr uint32_t kFrom = TableScaleFrom<FMT>::value, kSpan = 0x7F80u - kFrom;
+                careful0 = careful1 = (!unit0 && (m0 - kFrom) >= kSpan) || (!unit1 && (m1 - kFrom) >= kSpan);
+                const uint32_t m = (q & 2) ? m1 : m0;
+                const uint32_t t = tab[((q & 1) << 7) + (m & 0x7Fu)];
+                r = __uint_as_float(t + (m & 0x7F80u) * ((q & 1) ? 0xFFFF0000u : 0x00010000u));
+            } else {
+                const float a = __uint_as_float(((q & 2) ? m1 : m0) << 16);
+                r = __fdiv_rn((q & 1) ? Q : a, (q & 1) ? a : Q);
+            }
             inv0 = __shfl_sync(0xFFFFFFFFu, r, (lane & 28) | 1);
             inv1 = __shfl_sync(0xFFFFFFFFu, r, (lane & 28) | 3);
             inv0 = unit0 ? 1.0f : inv0;
@@ -355,7 +392,8 @@ __device__ __forceinline__ void careful_pair_fixup(const uint16_t *xa, const uin
 template <int FMT, bool CODES, bool SUMS>
 __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, uint8_t *__restrict__ codes,
                                               float *__restrict__ scales, float *__restrict__ row_rms, int64_t cols,
-                                              int64_t ld, int64_t r0, int64_t r1, float *sm_blocksum, int prefetch)
+                                              int64_t ld, int64_t r0, int64_t r1, float *sm_blocksum, int prefetch,
+                                              const uint32_t *tab)
 {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, q = lane & 3;
     const uint32_t nb = (uint32_t)(cols >> 6), cpr = (uint32_t)(cols >> 4);
@@ -394,7 +432,7 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
                 uint4 qa, qb;
                 float s, ss;
                 bool careful = false;
-                process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful);
+                process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful, tab);
                 if (CODES) {
                     *reinterpret_cast<uint4 *>(cp) = qa;
                     *reinterpret_cast<uint4 *>(cp + kCodecThreads * 16) = qb;
@@ -436,7 +474,7 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
             uint4 qa, qb;
             float s, ss;
             bool careful = false;
-            process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful);
+            process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful, tab);
             if (CODES) {
                 if (va) *reinterpret_cast<uint4 *>(cb_ + (size_t)ca * 16) = qa;
                 if (vb) *reinterpret_cast<uint4 *>(cb_ + (size_t)cb * 16) = qb;

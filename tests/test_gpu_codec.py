@@ -50,6 +50,23 @@ def test_every_bf16_pattern(fmt):
     check_roundtrip(rng.permutation(bits.reshape(-1)).reshape(64, 1024), fmt)
 
 
+@pytest.mark.parametrize("fmt", [api.FMT_E4M3FN_BLK, api.FMT_INT8_BLK])
+def test_every_block_absmax(fmt):
+    """One block per finite bf16 magnitude as its absmax (all 32 640 of them, either sign), the other elements
+    spread below it: the scale, its reciprocal and every code must match the oracle's IEEE divisions bit for bit
+    over the whole exponent range (unit-scale blocks, the subnormal-scale band and the table range)."""
+    rng = np.random.default_rng(11)
+    amax = np.arange(0, 0x7F80, dtype=np.uint32)
+    nblk = len(amax)
+    frac = rng.integers(0, 0x0400, size=(nblk, 64), dtype=np.uint32)          # up to 8 binades below the absmax
+    mag = np.maximum(amax[:, None].astype(np.int64) - frac, 0).astype(np.uint32)
+    pos = rng.integers(0, 64, nblk)
+    mag[np.arange(nblk), pos] = amax
+    sign = rng.integers(0, 2, size=(nblk, 64), dtype=np.uint32) << 15
+    x = (mag | sign).astype(np.uint16).reshape(nblk // 16, 1024)                  # 2040 rows of 16 blocks
+    check_roundtrip(x, fmt)
+
+
 def test_every_code_decodes():
     codes = np.arange(256, dtype=np.uint32).astype(np.uint8).reshape(4, 64)
     for fmt in FMTS:
