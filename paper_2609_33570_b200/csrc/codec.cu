@@ -29,12 +29,10 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     __shared__ uint32_t sm_tab[2][kScaleTableWords]; // scale tables: [0] Q = 448, [1] Q = 127
     if (FMT < 0 || FMT == HILORE_FMT_E4M3FN_BLK) fill_scale_table<HILORE_FMT_E4M3FN_BLK>(sm_tab[0]);
     if (FMT < 0 || FMT == HILORE_FMT_INT8_BLK) fill_scale_table<HILORE_FMT_INT8_BLK>(sm_tab[1]);
-    __syncthreads();
+    __syncthreads(); // scale tables are filled
     JobCursor cur;
-    Job j;
-    while (next_job(wk, cur, j)) {
-        if (j.op == OP_RECOVER)
-            continue;
+    DirectJob j;
+    while (next_job_direct(wk, cur, j)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
         if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
         else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
@@ -55,16 +53,17 @@ template <int FMT> __device__ __forceinline__ void recover_unit(const hilore_uni
 template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_kernel(const __grid_constant__ CodecWork wk)
 {
     __shared__ __align__(128) uint8_t sm_out[kRecoverStageBytes];
+    __shared__ UnitStage stage;
+    stage_units(wk, true, stage);
+    __syncthreads();
     uint32_t tile = 0;
     JobCursor cur;
     Job j;
-    while (next_job(wk, cur, j)) {
-        if (j.op != OP_RECOVER)
-            continue;
-        const int fmt = FMT >= 0 ? FMT : j.u.fmt;
-        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
-        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
-        else recover_unit<HILORE_FMT_INT8_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+    while (next_job(wk, stage, cur, j)) {
+        const int fmt = FMT >= 0 ? FMT : j.u->fmt;
+        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(*j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(*j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        else recover_unit<HILORE_FMT_INT8_BLK>(*j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
     }
     if (threadIdx.x == 0)
         bulk_wait_all(); // every bulk store of this CTA is complete before it gives up its shared memory
@@ -238,15 +237,10 @@ extern "C" int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit
     if (units_dev == nullptr || units_host == nullptr || avail == nullptr || action_io == nullptr)
         return HILORE_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int64_t total_rows = 0;
-    int common_fmt = units_host[0].fmt;
     for (int u = 0; u < U; ++u) {
         const int s = check_unit(units_host[u], false, false, false, false);
         if (s != HILORE_OK)
             return s;
-        total_rows += units_host[u].rows;
-        if (units_host[u].fmt != common_fmt)
-            common_fmt = -1;
     }
     if (phase == HILORE_PHASE_DECIDE) {
         if (exposure != nullptr && (kappa == nullptr || ebar == nullptr))
@@ -255,11 +249,25 @@ extern "C" int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit
                                               psi, recompute, retained_bytes);
         return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
     }
-    CodecWork wk{};
-    wk.units = units_dev;
-    wk.U = U;
-    wk.phase = phase;
-    wk.avail = avail;
-    wk.action = action_io;
-    return launch_codec(wk, total_rows, common_fmt, phase == HILORE_PHASE_RECOVER, st);
+    // one launch per slice of at most kStageUnits units (the kernels stage a slice's descriptors in shared memory)
+    for (int u0 = 0; u0 < U; u0 += kStageUnits) {
+        const int cnt = U - u0 < kStageUnits ? U - u0 : kStageUnits;
+        int64_t slice_rows = 0;
+        int slice_fmt = units_host[u0].fmt;
+        for (int u = u0; u < u0 + cnt; ++u) {
+            slice_rows += units_host[u].rows;
+            if (units_host[u].fmt != slice_fmt)
+                slice_fmt = -1;
+        }
+        CodecWork wk{};
+        wk.units = units_dev + u0;
+        wk.U = cnt;
+        wk.phase = phase;
+        wk.avail = avail + u0;
+        wk.action = action_io + u0;
+        const int s = launch_codec(wk, slice_rows, slice_fmt, phase == HILORE_PHASE_RECOVER, st);
+        if (s != HILORE_OK)
+            return s;
+    }
+    return HILORE_OK;
 }

@@ -53,8 +53,49 @@ __device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
 // every CTA takes the same share of every segment: rows [n*c/nC, n*(c+1)/nC) of its n rows.  All CTAs
 // therefore work inside one window of memory at a time and finish together -- measured faster on B200 than
 // giving each CTA one large private slice of a unit or of the whole launch.
+//
+// With a microbatch of 84 units a CTA meets a new unit every few iterations, so what it costs to get to the
+// next unit counts: the descriptors and the gating decisions of a launch (at most kStageUnits units; the host
+// cuts longer tables into several launches) are staged in shared memory once, and a CTA's share of n rows is
+// (n * K) >> 32 with K = floor(c * 2^32 / nC) computed once per kernel -- the same partition for all CTAs
+// (consecutive CTAs share their boundary, the last one ends at n) for one multiplication instead of two 64-bit
+// divisions per unit.
+constexpr int kStageUnits = 96;
+
+struct UnitStage {
+    hilore_unit u[kStageUnits];
+    int op[kStageUnits];
+    uint64_t k0, k1; // floor(c * 2^32 / nC), floor((c + 1) * 2^32 / nC) for this CTA c
+};
+
+// Stage the launch's units: what to do with each (OP_NONE if the launch is not gated into it or it lacks a
+// buffer the operation needs) and its descriptor.  `recover`: which of the two kernels is asking.
+__device__ __forceinline__ void stage_units(const CodecWork &wk, bool recover, UnitStage &st)
+{
+    if (threadIdx.x == 0) {
+        st.k0 = ((uint64_t)blockIdx.x << 32) / gridDim.x;
+        st.k1 = ((uint64_t)(blockIdx.x + 1) << 32) / gridDim.x;
+    }
+    for (int t = threadIdx.x; t < wk.U; t += blockDim.x) {
+        int op = unit_op(wk, t);
+        if (recover ? (op != OP_RECOVER) : (op != OP_COMPRESS && op != OP_STATS))
+            op = OP_NONE;
+        if (op != OP_NONE) {
+            hilore_unit u = wk.units ? wk.units[t] : wk.single;
+            const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
+            if ((op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (op == OP_STATS && (!u.x || !u.row_rms)) ||
+                (op == OP_RECOVER && (!u.out || !u.codes || (scaled && !u.scales))))
+                op = OP_NONE; // the unit lacks a buffer this operation needs: leave it untouched
+            if (op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
+                u.row_rms = nullptr; // token magnitudes were collected at capture time
+            st.u[t] = u;
+        }
+        st.op[t] = op;
+    }
+}
+
 struct Job {
-    hilore_unit u;
+    const hilore_unit *u; // in the shared-memory stage
     int op;
     int64_t r0, r1; // this CTA's rows of the current segment
 };
@@ -64,21 +105,61 @@ struct JobCursor {
     int64_t seg_row = 0; // first row of the next segment of unit ui
 };
 
-__device__ __forceinline__ bool next_job(const CodecWork &wk, JobCursor &cur, Job &j)
+__device__ __forceinline__ bool next_job(const CodecWork &wk, const UnitStage &st, JobCursor &cur, Job &j)
+{
+    for (; cur.ui < wk.U; ++cur.ui, cur.seg_row = 0) {
+        j.op = st.op[cur.ui];
+        if (j.op == OP_NONE)
+            continue;
+        j.u = &st.u[cur.ui];
+        const hilore_unit &u = *j.u;
+        // equal segments, as close to seg_bytes each as the unit's size allows
+        const int64_t unit_bytes = u.rows * u.cols * 2;
+        int64_t seg_rows = u.rows;
+        if (unit_bytes >= wk.seg_bytes + wk.seg_bytes / 2) {
+            const int64_t nseg = (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes;
+            seg_rows = (u.rows + nseg - 1) / nseg;
+        }
+        seg_rows = max((int64_t)gridDim.x, seg_rows);
+        while (cur.seg_row < u.rows) {
+            const int64_t s0 = cur.seg_row, n = min(seg_rows, u.rows - s0);
+            cur.seg_row += n;
+            if (n < (1ll << 31)) {
+                j.r0 = s0 + (int64_t)(((uint64_t)n * st.k0) >> 32);
+                j.r1 = s0 + (int64_t)(((uint64_t)n * st.k1) >> 32);
+            } else {
+                j.r0 = s0 + (n * (int64_t)blockIdx.x) / gridDim.x;
+                j.r1 = s0 + (n * (int64_t)(blockIdx.x + 1)) / gridDim.x;
+            }
+            if (j.r0 < j.r1)
+                return true; // the cursor already points at the next segment
+        }
+    }
+    return false;
+}
+
+// The same walk without the stage: descriptors and gates are read from global memory at every unit.  The
+// compress kernel uses this form -- its 64-register budget is full, and the staged form costs it more in
+// register traffic inside the hot loop than it saves per unit.
+struct DirectJob {
+    hilore_unit u;
+    int op;
+    int64_t r0, r1;
+};
+
+__device__ __forceinline__ bool next_job_direct(const CodecWork &wk, JobCursor &cur, DirectJob &j)
 {
     for (; cur.ui < wk.U; ++cur.ui, cur.seg_row = 0) {
         j.op = unit_op(wk, cur.ui);
-        if (j.op == OP_NONE)
+        if (j.op != OP_COMPRESS && j.op != OP_STATS)
             continue;
         j.u = wk.units ? wk.units[cur.ui] : wk.single;
         const hilore_unit &u = j.u;
         const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
-        if ((j.op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (j.op == OP_STATS && (!u.x || !u.row_rms)) ||
-            (j.op == OP_RECOVER && (!u.out || !u.codes || (scaled && !u.scales))))
+        if ((j.op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (j.op == OP_STATS && (!u.x || !u.row_rms)))
             continue; // the unit lacks a buffer this operation needs: leave it untouched
         if (j.op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
             j.u.row_rms = nullptr; // token magnitudes were collected at capture time
-        // equal segments, as close to seg_bytes each as the unit's size allows
         const int64_t unit_bytes = u.rows * u.cols * 2;
         const int64_t nseg = max((int64_t)1, (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes);
         const int64_t seg_rows = max((int64_t)gridDim.x, (u.rows + nseg - 1) / nseg);

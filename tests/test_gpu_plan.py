@@ -158,3 +158,46 @@ def test_units_without_buffers_are_skipped_and_bad_tables_rejected():
                                  check=False) == api.SHAPE
     assert api.hilore_plan_apply(dev, host, 1, 9, None, None, None, 0, 0, avail, action, None, None, None,
                                  check=False) == api.INVALID_ARG
+
+
+def test_tables_longer_than_one_launch_slice():
+    """210 small units (more than the kernels stage per launch) with mixed formats and gates: CAPTURE then RECOVER
+    must touch exactly the gated units, whichever slice of the table they fall into."""
+    rng = np.random.default_rng(17)
+    U = 210
+    fmts = [(api.FMT_E4M3FN_BLK, api.FMT_E4M3FN_RAW, api.FMT_INT8_BLK)[i % 3] for i in range(U)]
+    shapes = [((5, 64), (3, 192), (9, 128), (2, 1536))[i % 4] for i in range(U)]
+    q = [(L, H, R, L, L)[i % 5] for i in range(U)]
+    xs = [synth.activation_unit(rng, r, c) for r, c in shapes]
+    bufs, units = [], []
+    for x, (r, c), f in zip(xs, shapes, fmts):
+        b = dict(x=G.dev(x), codes=G.Guarded(r * c), scales=G.Guarded(r * (c // 64) * 4), out=G.Guarded(r * c * 2),
+                 rms=G.Guarded(r * 4))
+        bufs.append(b)
+        units.append(dict(x=b["x"], codes=b["codes"].ptr(), scales=None if f == api.FMT_E4M3FN_RAW else b["scales"].ptr(),
+                          out=b["out"].ptr(), row_rms=b["rms"].ptr(), rows=r, cols=c, fmt=f,
+                          block=0 if f == api.FMT_E4M3FN_RAW else 64))
+    dev, host = api.make_unit_table(units)
+    avail = G.dev(np.asarray(q, np.uint8))
+    action = G.dev(np.asarray(q, np.uint8))                # every L candidate is decoded again
+    api.hilore_plan_apply(dev, host, U, api.PHASE_CAPTURE, None, None, None, 0, 0, avail, action, None, None, None)
+    api.hilore_plan_apply(dev, host, U, api.PHASE_RECOVER, None, None, None, 0, 0, avail, action, None, None, None)
+    canary = G.CANARY | (G.CANARY << 8)
+    for i, (x, (r, c), f, b) in enumerate(zip(xs, shapes, fmts, bufs)):
+        blk = 0 if f == api.FMT_E4M3FN_RAW else 64
+        codes, out, rms = b["codes"].numpy(np.uint8, (r, c)), b["out"].numpy(np.uint16, (r, c)), b["rms"].numpy(np.float32, (r,))
+        if q[i] == L:
+            oc, osc = oracle.compress(x, f, blk)
+            assert np.array_equal(codes, oc), i
+            if blk:
+                assert np.array_equal(b["scales"].numpy(np.float32, (r, c // 64)), osc), i
+            orec = oracle.recover(oc, osc, f, blk)
+            nan = (orec & 0x7FFF) > 0x7F80
+            assert np.array_equal(out[~nan], orec[~nan]), i
+            assert G.rel_err(rms, oracle.row_rms(x)).max() <= 1e-5
+        else:
+            assert np.all(codes == G.CANARY) and np.all(out == canary), i
+            if q[i] == H:
+                assert G.rel_err(rms, oracle.row_rms(x)).max() <= 1e-5
+            else:
+                assert np.all(b["rms"].numpy(np.uint8, (r * 4,)) == G.CANARY), i
