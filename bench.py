@@ -34,10 +34,10 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per algorithmic byte of the two codec kernels, from the ncu captures
 # summarised in profiles/codec_kernels_bench_1p5B_and_unit8192x8960.md (one unit [8192, 8960], 224.8 MB
 # algorithmic; traffic grows in proportion to the elements processed).  Reads match the algorithmic
-# reads (compress 1.04x, recover 1.00x); the write side of that small capture is low because about a
+# reads (compress 1.02x, recover 1.00x); the write side of that small capture is low because about a
 # third of the written bytes was still dirty in L2 when the kernel ended.
-DRAM_PER_ALGORITHMIC = {"compress": (153.273088 + 51.505664) / 224.822,
-                        "recover": (78.084096 + 89.138944) / 224.789}
+DRAM_PER_ALGORITHMIC = {"compress": (150.173696 + 44.848640) / 224.822,
+                        "recover": (78.083072 + 91.620352) / 224.789}
 
 
 # ---------------------------------------------------------------- accounting (bytes the method must move)
