@@ -300,3 +300,20 @@ def test_blk_unit_scale_threshold(fmt, Q, last_unit):
             assert s[0, 0] == 1.0 and np.all(c == 0)
         else:
             assert s[0, 0] == np.float32(amax) / np.float32(Q) and (c[0, 7] & 0x7F) == (0x7E if fmt == FMT_E4M3FN_BLK else 127)
+
+
+def test_unscaled_tables_match_the_recorded_digests():
+    """The exhaustive encode / decode tables of the oracle hash to the digests recorded from the cast the paper
+    names (a fixed pin that does not depend on the torch installed next to the tests)."""
+    import hashlib
+    want = {}
+    for line in open(os.path.join(GOLD, "e4m3fn_table_digests.txt")):
+        if not line.startswith("#") and "|" in line:
+            k, v = (p.strip() for p in line.split("|"))
+            want[k] = v
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16).reshape(1024, 64)
+    codes, _ = oracle.compress(bits, 0, 0)
+    assert hashlib.sha256(codes.tobytes()).hexdigest() == want["encode"]
+    every = np.arange(256, dtype=np.uint32).astype(np.uint8).reshape(4, 64)
+    rec = oracle.recover(every, None, 0, 0)
+    assert hashlib.sha256(rec.astype("<u2").tobytes()).hexdigest() == want["decode"]
