@@ -184,3 +184,18 @@ def test_exposure_from_fused_token_rms():
     o_rms = np.stack([oracle.row_rms(x) for x in units])
     oE, _ = oracle.unit_exposure(omega, ro.mask, o_rms)
     assert G.rel_err(E, oE).max() <= RTOL
+
+
+def test_ratio_over_the_whole_exponent_range():
+    """Log-ratio from -80 to +80 (r from 1e-35 to 5e34): ratio and omega stay within 1e-5 of the oracle."""
+    ro = synth.rollout(41, 4, 4, 1024, rewards="uniform")
+    d = np.linspace(-80.0, 80.0, ro.logp_new.size, dtype=np.float32).reshape(ro.logp_new.shape)
+    ro.logp_old[:] = ro.logp_new - d
+    got = G.grpo_coeffs(ro, N_norm=ro.n_valid)
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, r, chi = oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, None, ro.mask, N_norm=ro.n_valid)
+    assert G.rel_err(got["ratio"], r).max() <= RTOL
+    hi, lo = np.float32(1.2), np.float32(0.8)
+    near = (np.abs(r - hi) <= 4 * np.spacing(hi)) | (np.abs(r - lo) <= 4 * np.spacing(lo))
+    assert np.array_equal(got["chi"][~near], chi[~near])
+    assert G.rel_err(got["omega"][~near], w[~near]).max() <= RTOL
