@@ -124,9 +124,11 @@ __device__ __forceinline__ float exp_ratio(float d)
 template <bool KL, bool EXTRA, int VAR>
 __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid_constant__ CoeffArgs a)
 {
-    const int64_t tile = blockIdx.x;
-    const int64_t row = tile / a.tiles_per_row;
-    const int tt = (int)(tile - row * a.tiles_per_row);
+    // 32-bit index arithmetic (the host checks that the grid fits)
+    const uint32_t tpr = (uint32_t)a.tiles_per_row;
+    const uint32_t row32 = tpr == 1 ? blockIdx.x : blockIdx.x / tpr;
+    const int tt = (int)(blockIdx.x - row32 * tpr);
+    const int64_t row = row32;
     const int tid = threadIdx.x, lane = tid & 31;
     const int64_t rowbase = row * a.T;
 
