@@ -29,10 +29,15 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     __shared__ uint32_t sm_tab[2][kScaleTableWords]; // scale tables: [0] Q = 448, [1] Q = 127
     if (FMT < 0 || FMT == HILORE_FMT_E4M3FN_BLK) fill_scale_table<HILORE_FMT_E4M3FN_BLK>(sm_tab[0]);
     if (FMT < 0 || FMT == HILORE_FMT_INT8_BLK) fill_scale_table<HILORE_FMT_INT8_BLK>(sm_tab[1]);
-    __syncthreads(); // scale tables are filled
+    __shared__ uint64_t sm_share[2]; // this CTA's multipliers for its share of a unit's rows
+    if (threadIdx.x == 0) {
+        sm_share[0] = ((uint64_t)blockIdx.x << 32) / gridDim.x;
+        sm_share[1] = ((uint64_t)(blockIdx.x + 1) << 32) / gridDim.x;
+    }
+    __syncthreads(); // scale tables and shares are filled
     JobCursor cur;
     DirectJob j;
-    while (next_job_direct(wk, cur, j)) {
+    while (next_job_direct(wk, cur, j, sm_share)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
         if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
         else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);

@@ -147,7 +147,7 @@ struct DirectJob {
     int64_t r0, r1;
 };
 
-__device__ __forceinline__ bool next_job_direct(const CodecWork &wk, JobCursor &cur, DirectJob &j)
+__device__ __forceinline__ bool next_job_direct(const CodecWork &wk, JobCursor &cur, DirectJob &j, const uint64_t *share)
 {
     for (; cur.ui < wk.U; ++cur.ui, cur.seg_row = 0) {
         j.op = unit_op(wk, cur.ui);
@@ -161,13 +161,22 @@ __device__ __forceinline__ bool next_job_direct(const CodecWork &wk, JobCursor &
         if (j.op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
             j.u.row_rms = nullptr; // token magnitudes were collected at capture time
         const int64_t unit_bytes = u.rows * u.cols * 2;
-        const int64_t nseg = max((int64_t)1, (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes);
-        const int64_t seg_rows = max((int64_t)gridDim.x, (u.rows + nseg - 1) / nseg);
+        int64_t seg_rows = u.rows;
+        if (unit_bytes >= wk.seg_bytes + wk.seg_bytes / 2) {
+            const int64_t nseg = (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes;
+            seg_rows = (u.rows + nseg - 1) / nseg;
+        }
+        seg_rows = max((int64_t)gridDim.x, seg_rows);
         while (cur.seg_row < u.rows) {
             const int64_t s0 = cur.seg_row, n = min(seg_rows, u.rows - s0);
             cur.seg_row += n;
-            j.r0 = s0 + (n * (int64_t)blockIdx.x) / gridDim.x;
-            j.r1 = s0 + (n * (int64_t)(blockIdx.x + 1)) / gridDim.x;
+            if (n < (1ll << 31)) { // share[0..1] = floor(c * 2^32 / nC), floor((c + 1) * 2^32 / nC)
+                j.r0 = s0 + (int64_t)(((uint64_t)n * share[0]) >> 32);
+                j.r1 = s0 + (int64_t)(((uint64_t)n * share[1]) >> 32);
+            } else {
+                j.r0 = s0 + (n * (int64_t)blockIdx.x) / gridDim.x;
+                j.r1 = s0 + (n * (int64_t)(blockIdx.x + 1)) / gridDim.x;
+            }
             if (j.r0 < j.r1)
                 return true; // the cursor already points at the next segment
         }
