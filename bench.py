@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 # algorithmic; traffic grows in proportion to the elements processed).  Reads match the algorithmic
 # reads (compress 1.02x, recover 1.00x); the write side of that small capture is low because about a
 # third of the written bytes was still dirty in L2 when the kernel ended.
-DRAM_PER_ALGORITHMIC = {"compress": (150.173696 + 44.848640) / 224.822,
-                        "recover": (78.083072 + 91.620352) / 224.789}
+DRAM_PER_ALGORITHMIC = {"compress": (150.254592 + 45.741568) / 224.822,
+                        "recover": (78.083072 + 89.875712) / 224.789}
 
 
 # ---------------------------------------------------------------- accounting (bytes the method must move)
