@@ -319,9 +319,9 @@ typedef struct hilore_unit {
 
 /*
  * Risk score, H / L / R gating and the batched capture / encode / recover of all units of a microbatch
- * in ONE launch per phase (Eq. "token-weighted-risk": psi_u = kappa_c(u) E_u ebar_u;
- * Eq. "available-recovery-actions").  All decisions stay on the device: the gating arrays are read
- * by the kernels, so no phase needs a host synchronisation.
+ * in ONE launch per phase and 96 units (a longer table runs as consecutive launches over slices of 96)
+ * (Eq. "token-weighted-risk": psi_u = kappa_c(u) E_u ebar_u; Eq. "available-recovery-actions").  All decisions
+ * stay on the device: the gating arrays are read by the kernels, so no phase needs a host synchronisation.
  *
  *   units_dev   [U] hilore_unit on the DEVICE.     units_host  the same table on the HOST (read during
  *               the call for validation and launch sizing; must match units_dev).
