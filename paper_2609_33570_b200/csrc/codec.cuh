@@ -8,8 +8,9 @@
 // squares of a batch fit in shared memory; at the end of a batch each warp adds the blocks of whole
 // rows in a fixed order, so the token RMS is deterministic (no floating-point atomics anywhere).
 // The instruction budget matters: at 6.5 TB/s the SM has about 8 issue slots per element, so the hot
-// loop uses packed bf16x2 maxima, packed f32x2 multiplies / FMAs, one IEEE division per thread and
-// pair of blocks, and pointer increments instead of index arithmetic.
+// loop uses packed bf16x2 maxima, packed f32x2 multiplies / FMAs, a 128-entry table in place of the two IEEE
+// divisions of a block, one conversion block per four codes, a rare-path repair after the stores instead of
+// calls inside the loop, and pointer increments instead of index arithmetic.
 #pragma once
 
 #include "common.cuh"
@@ -358,9 +359,9 @@ __device__ __forceinline__ void chunk_pass(const uint32_t (&w)[8], float inv, ui
 
 // Everything a thread does with the two chunks it holds.  All 32 lanes must call this together
 // (xor-shuffles inside).  The four lanes of a quad hold one 64-element block per chunk.
-//   CODES: the two IEEE divisions of a block (s = amax / Q, inv = Q / amax) are spread over the quad:
-//          lanes 0 / 1 compute s / inv of chunk 0's block, lanes 2 / 3 those of chunk 1's block -- one
-//          division per thread instead of four.  `s_store` is the scale of chunk 0's block in lanes with
+//   CODES: the two quotients of a block (s = amax / Q, inv = Q / amax; IEEE divisions, or with LATER the scale
+//          table) are spread over the quad: lanes 0 / 1 compute s / inv of chunk 0's block, lanes 2 / 3 those
+//          of chunk 1's block -- one per thread instead of four.  `s_store` is the scale of chunk 0's block in lanes with
 //          (lane & 3) == 0 and of chunk 1's block in lanes with (lane & 3) == 2.
 //   SUMS:  `bsum` is the block sum of squares of chunk 0's block in even lanes, of chunk 1's in odd lanes.
 //   LATER: blocks that need the careful rules (Inf, NaN, overflow of the unscaled cast) are only reported in
