@@ -343,7 +343,7 @@ __device__ __forceinline__ void chunk_pass(const uint32_t (&w)[8], float inv, ui
             f32x2_unpack(xa, a0, a1);
             f32x2_unpack(xb, b0, b1);
             if (FMT == HILORE_FMT_INT8_BLK)
-                cw[i] = int8_code(a0) | (int8_code(a1) << 8) | (int8_code(b0) << 16) | (int8_code(b1) << 24);
+                cw[i] = cvt_s8x4(a0, a1, b0, b1); // |q| <= 127 (1 + 2^-23) here, so saturation at -128 cannot occur
             else
                 cw[i] = cvt_e4m3x4(a0, a1, b0, b1);
         }

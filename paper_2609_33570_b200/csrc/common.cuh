@@ -71,6 +71,15 @@ __device__ __forceinline__ uint32_t cvt_e4m3x4(float x0, float x1, float x2, flo
     return r;
 }
 
+// Four fp32 -> four int8 codes in one word (round to nearest even, saturating), x0 in the lowest byte.
+__device__ __forceinline__ uint32_t cvt_s8x4(float x0, float x1, float x2, float x3)
+{
+    uint32_t hi, r;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(__float2int_rn(x3)), "r"(__float2int_rn(x2)), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(__float2int_rn(x1)), "r"(__float2int_rn(x0)), "r"(hi));
+    return r;
+}
+
 // Two E4M3FN codes (low 16 bits of `c`) -> two fp16 (exact), packed.
 __device__ __forceinline__ uint32_t cvt_e4m3x2_to_f16x2(uint32_t c)
 {
