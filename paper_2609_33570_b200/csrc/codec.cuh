@@ -609,10 +609,8 @@ template <int FMT> __device__ __forceinline__ void decode16(const uint4 cd, floa
             const uint32_t two = p ? (cw[i] >> 16) : (cw[i] & 0xFFFFu); // two codes
             float f0, f1;
             if (FMT == HILORE_FMT_INT8_BLK) {
-                const int b0 = (int)(int8_t)(two & 0xFF), b1 = (int)(int8_t)(two >> 8);
-                const float qnan = __uint_as_float(0x7FC00000u);
-                f0 = (b0 == -128) ? qnan : (float)b0;
-                f1 = (b1 == -128) ? qnan : (float)b1;
+                f0 = (float)(int)(int8_t)(two & 0xFF);
+                f1 = (float)(int)(int8_t)(two >> 8);
             } else {
                 const uint32_t hh = cvt_e4m3x2_to_f16x2(two);
                 f0 = f16_lo_to_f32(hh);
@@ -623,6 +621,14 @@ template <int FMT> __device__ __forceinline__ void decode16(const uint4 cd, floa
                 f32x2_unpack(y, f0, f1);
             }
             o[2 * i + p] = cvt_bf16x2(f1, f0);
+        }
+        if (FMT == HILORE_FMT_INT8_BLK) { // code 0x80 is the reserved NaN: rare, patched per word
+            const uint32_t is_nan = __vcmpeq4(cw[i], 0x80808080u); // 0xFF in every byte that holds 0x80
+            if (is_nan) {
+                const uint32_t lo = __byte_perm(is_nan, 0, 0x1100), hi = __byte_perm(is_nan, 0, 0x3322);
+                o[2 * i] = (o[2 * i] & ~lo) | (0x7FC07FC0u & lo);
+                o[2 * i + 1] = (o[2 * i + 1] & ~hi) | (0x7FC07FC0u & hi);
+            }
         }
     }
 }
