@@ -109,11 +109,15 @@ def test_allocate_consumes_device_side_risk_scores():
                           None, None)
     dtau = np.tile(np.array([0.0, 2.0, 1.5]), (U, 1))
     dmem = np.tile(np.array([0.0, 16384.0, 8704.0]), (U, 1))
-    M_res, delta_b = 3.2 * 16384, float(psi.sum().item() * 0.5)
+    # the oracle's own psi from the host inputs; the device's must be the same bits
+    _, o_psi, _, _ = oracle.plan(exposure.cpu().numpy(), np.ones(U, np.float32), np.full(U, 0.025, np.float32), 0.0,
+                                 float("inf"), [H] * U, [64] * U, [128] * U, [1] * U, [64] * U)
+    assert np.array_equal(psi.cpu().numpy().view(np.uint32), o_psi.view(np.uint32))
+    M_res, delta_b = 3.2 * 16384, float(o_psi.astype(np.float64).sum() * 0.5)
     nws = api.hilore_allocate_workspace_bytes(U, 1024)
     ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
     api.hilore_allocate(U, psi, torch.from_numpy(dtau).cuda(), torch.from_numpy(dmem).cuda(), avail, M_res, delta_b, 1024,
                         action, None, None, ws, nws)
-    oa, _ = oracle.allocate(psi.cpu().numpy(), dtau, dmem, avail.cpu().numpy(), M_res, delta_b)
+    oa, _ = oracle.allocate(o_psi, dtau, dmem, np.full(U, H, np.uint8), M_res, delta_b)
     assert np.array_equal(action.cpu().numpy(), oa)
     assert (oa == L).sum() >= 1 and (oa == H).sum() >= 1

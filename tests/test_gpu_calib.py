@@ -28,7 +28,8 @@ def test_relative_error_of_the_round_trip(fmt, rows, cols):
     codes, scales, _ = G.compress(x, fmt)
     xh = G.recover(codes, scales, fmt)
     e, n2 = rel_error_gpu(x, xh)
-    want = oracle.relative_error(x, xh)
+    o_codes, o_scales = oracle.compress(x, fmt)[:2]           # the oracle's own round trip
+    want = oracle.relative_error(x, oracle.recover(o_codes, o_scales, fmt))
     assert e == pytest.approx(want, rel=1e-6)
     xf = (x.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     assert n2[1] == pytest.approx((xf ** 2).sum(), rel=1e-6)

@@ -152,4 +152,7 @@ def test_error_statistic_of_gpu_roundtrip_matches_oracle():
     x = synth.activation_unit(np.random.default_rng(9), 256, 1536)
     codes, _, _ = G.compress(x, api.FMT_E4M3FN_RAW)
     rec = G.recover(codes, None, api.FMT_E4M3FN_RAW)
-    assert oracle.relative_error(x, rec) == oracle.relative_error(x, oracle.recover(codes, None, 0, 0))
+    o_codes, _ = oracle.compress(x, api.FMT_E4M3FN_RAW, 0)
+    o_rec = oracle.recover(o_codes, None, 0, 0)
+    assert np.array_equal(codes, o_codes) and np.array_equal(rec, o_rec)
+    assert 0.02 < oracle.relative_error(x, o_rec) < 0.035

@@ -35,11 +35,19 @@ def coeffs(ro, beta=0.0, variant=None):
             chi.numpy(np.uint8, (n_rows, T)))
 
 
+def oracle_record(ro):
+    """adv, omega, ratio of a rollout from the oracle (host inputs only)."""
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, r, _ = oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, None, ro.mask, N_norm=ro.n_valid)
+    return adv, w, r
+
+
 @pytest.mark.parametrize("P,G_,T,lengths", [(4, 8, 256, "full"), (64, 8, 1024, "uniform"), (3, 4, 52, "uniform")])
 def test_diagnostics_match_oracle(P, G_, T, lengths):
+    """The same record (written by the oracle from host inputs) through both diagnostics: counts exact."""
     ro = synth.rollout(7, P, G_, T, rewards="bernoulli", lengths=lengths, min_len=8)
     ro.logp_old[:] = ro.logp_new + np.random.default_rng(1).normal(0, 0.15, ro.logp_new.shape).astype(np.float32)
-    adv, omega, ratio, chi = coeffs(ro)
+    adv, omega, ratio = oracle_record(ro)
     counts, share, total = diag_gpu(adv, ratio, ro.mask, omega)
     oc, oshare, ototal = oracle.omega_diagnostics(adv, ratio, ro.mask, omega)
     assert counts.tolist() == oc.tolist()
@@ -47,6 +55,23 @@ def test_diagnostics_match_oracle(P, G_, T, lengths):
     assert counts[3] == counts[0] + counts[1] + counts[2]                 # Remark 1 accounting at beta = 0
     a = diag_gpu(adv, ratio, ro.mask, omega)
     assert a[1] == share and a[2] == total                                  # deterministic
+
+
+def test_diagnostics_of_the_gpu_record_end_to_end():
+    """GPU coefficients -> GPU diagnostics against oracle coefficients -> oracle diagnostics.  The log-ratios keep a
+    distance from the clip bounds, so that the two chains classify every slot alike."""
+    ro = synth.rollout(9, 32, 8, 512, rewards="bernoulli", lengths="uniform", min_len=8)
+    d = np.random.default_rng(2).normal(0, 0.15, ro.logp_new.shape).astype(np.float32)
+    for bound in (np.log(1.2), np.log(0.8)):
+        close = np.abs(d - bound) < 1e-3
+        d[close] += np.float32(4e-3)
+    ro.logp_old[:] = ro.logp_new - d
+    adv_g, omega_g, ratio_g, _ = coeffs(ro)
+    counts, share, total = diag_gpu(adv_g, ratio_g, ro.mask, omega_g)
+    adv, omega, ratio = oracle_record(ro)
+    oc, oshare, ototal = oracle.omega_diagnostics(adv, ratio, ro.mask, omega)
+    assert counts.tolist() == oc.tolist()
+    assert share == pytest.approx(oshare, rel=1e-5) and total == pytest.approx(ototal, rel=1e-5)
 
 
 def test_diagnostics_ties_and_degenerate_records():

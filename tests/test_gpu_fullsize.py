@@ -54,17 +54,22 @@ def test_bench_step_1p5B_shaped_microbatch():
     assert wl.retained.cpu().tolist() == want_bytes
     for u in (0, 1, 2, 41, 42, 43, 81, 82, 83):
         check_rows(wl.x[u], wl.codes[u], wl.scales[u], wl.out[u], wl.rms[u], sample_rows(rng, wl.rows), api.FMT_E4M3FN_BLK)
-    # coefficients of microbatch 3 and the exposure of all 84 units (token RMS as the GPU wrote it)
+    # coefficients of microbatch 3, then exposure, psi and action of a sample of units, every expected value from the
+    # oracle's own chain (its omega, its token RMS of the whole unit): a unit's exposure depends on that unit only
     ro = wl.ro
     sl = slice(3 * bench.MB_RESP, 4 * bench.MB_RESP)
     adv = oracle.group_advantages(ro.rewards, ro.G)
     w, _, _ = oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=ro.n_valid)
-    got_w = wl.omega.cpu().numpy()
-    assert G.rel_err(got_w, w).max() <= 1e-5
-    oE, _ = oracle.unit_exposure(got_w, ro.mask[sl], wl.rms.cpu().numpy())
-    assert G.rel_err(wl.exposure.cpu().numpy(), oE).max() <= 1e-5
-    psi = (wl.kappa.cpu().numpy() * wl.exposure.cpu().numpy()).astype(np.float32) * wl.ebar.cpu().numpy()
-    assert np.array_equal(wl.psi.cpu().numpy().view(np.uint32), psi.view(np.uint32))
+    assert G.rel_err(wl.omega.cpu().numpy(), w).max() <= 1e-5
+    sample = [0, 2, 41, 43, 83]
+    o_rms = np.stack([oracle.row_rms(bits(wl.x[u])) for u in sample])
+    oE, _ = oracle.unit_exposure(w, ro.mask[sl], o_rms)
+    assert G.rel_err(wl.exposure.cpu().numpy()[sample], oE).max() <= 1e-5
+    kappa, ebar = wl.kappa.cpu().numpy()[sample], wl.ebar.cpu().numpy()[sample]
+    oa, opsi, orec, oret = oracle.plan(oE, kappa, ebar, float("inf"), float("inf"), [L] * len(sample), [wl.shapes[u][0] for u in sample],
+                                       [wl.shapes[u][1] for u in sample], [1] * len(sample), [64] * len(sample))
+    assert G.rel_err(wl.psi.cpu().numpy()[sample], opsi).max() <= 1e-5
+    assert np.array_equal(wl.action.cpu().numpy()[sample], oa) and np.array_equal(wl.retained.cpu().numpy()[sample].view(np.uint64), oret)
     # every byte of every output was written: no canary left in a random sample of code rows
     for u in (5, 50):
         assert not bool((wl.scales[u] == 0).all())
@@ -115,19 +120,30 @@ def test_7B_shaped_mixed_plan():
     api.hilore_unit_exposure(omega, t(ro.mask[sl]), n_mb, 2048, rms, U, rows, 0, 1e-8, expo, None, ws, nws)
     kappa = torch.from_numpy(np.random.default_rng(3).uniform(0.5, 2.0, U).astype(np.float32)).to(dev)
     ebar = torch.full((U,), 0.0266, dtype=torch.float32, device=dev)
+    # thresholds at midpoints between order statistics of psi, so that no unit sits near a threshold
     E = expo.cpu().numpy()
-    oE, _ = oracle.unit_exposure(omega.cpu().numpy(), ro.mask[sl], rms.cpu().numpy())
-    assert G.rel_err(E, oE).max() <= 1e-5
     psi_h = (kappa.cpu().numpy() * E).astype(np.float32) * ebar.cpu().numpy()
     srt = np.sort(psi_h)
     lo, hi = float((srt[41] + srt[42]) / 2), float((srt[U - 26] + srt[U - 25]) / 2)
     call(api.PHASE_DECIDE, E=expo, kappa=kappa, ebar=ebar, lo=lo, hi=hi, psi=psi)
     a = action.cpu().numpy()
-    oa, opsi, orec, oret = oracle.plan(E, kappa.cpu().numpy(), ebar.cpu().numpy(), lo, hi, [H] * U, [s[0] for s in shapes],
-                                       [s[1] for s in shapes], [1] * U, [64] * U)
-    assert np.array_equal(a, oa) and np.array_equal(psi.cpu().numpy().view(np.uint32), opsi.view(np.uint32))
-    assert np.array_equal(rec.cpu().numpy(), orec) and np.array_equal(retained.cpu().numpy().view(np.uint64), oret)
     assert [(a == v).sum() for v in (L, H, R)] == [42, 25, 17]
+    assert np.array_equal(rec.cpu().numpy(), (a == R).astype(np.uint8))
+    # expected values of a sample of units from the oracle's own chain: its advantages and omega from the host
+    # inputs, its token RMS of the whole unit, its exposure, psi and action
+    adv_o = oracle.group_advantages(ro.rewards, 16)
+    w_o, _, _ = oracle.grpo_coeffs(adv_o[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=2048 * 128 * 16)
+    assert G.rel_err(omega.cpu().numpy(), w_o).max() <= 1e-5
+    sample = [0, 1, 40, 82, 5]                             # four narrow units and one wide one
+    o_rms = np.stack([oracle.row_rms(bits(x[u])) for u in sample])
+    oE, _ = oracle.unit_exposure(w_o, ro.mask[sl], o_rms)
+    assert G.rel_err(E[sample], oE).max() <= 1e-5
+    oa, opsi, orec, oret = oracle.plan(oE, kappa.cpu().numpy()[sample], ebar.cpu().numpy()[sample], lo, hi, [H] * len(sample),
+                                       [shapes[u][0] for u in sample], [shapes[u][1] for u in sample], [1] * len(sample),
+                                       [64] * len(sample))
+    assert G.rel_err(psi.cpu().numpy()[sample], opsi).max() <= 1e-5
+    assert np.array_equal(a[sample], oa) and np.array_equal(rec.cpu().numpy()[sample], orec)
+    assert np.array_equal(retained.cpu().numpy()[sample].view(np.uint64), oret)
     call(api.PHASE_ENCODE)
     call(api.PHASE_RECOVER)
     torch.cuda.synchronize()
@@ -173,7 +189,7 @@ def test_variable_length_rollout_batch_full_size():
     _, _, rms = G.compress(x, api.FMT_E4M3FN_BLK)
     om = np.ascontiguousarray(got["omega"][8:12])
     E, sw = G.unit_exposure(om, np.ascontiguousarray(ro.mask[8:12]), rms[None, :])
-    oE, osw = oracle.unit_exposure(om, np.ascontiguousarray(ro.mask[8:12]), oracle.row_rms(x)[None, :])
+    oE, osw = oracle.unit_exposure(np.ascontiguousarray(w[8:12]), np.ascontiguousarray(ro.mask[8:12]), oracle.row_rms(x)[None, :])
     assert G.rel_err(E, oE).max() <= 1e-5 and abs(sw - osw) <= 1e-5 * osw
 
 
