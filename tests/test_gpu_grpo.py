@@ -127,10 +127,16 @@ def _rms_for(ro, U, seed):
     return (rng.random((U, ro.n_resp * ro.T), dtype=np.float32) * np.float32(2) + np.float32(0.25))
 
 
+def oracle_omega(ro):
+    """Coefficients of a rollout from the oracle (host inputs only): the common input of both exposure paths."""
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    return oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, None, ro.mask, N_norm=ro.n_valid)[0]
+
+
 @pytest.mark.parametrize("U", [1, 2, 9, 84])
 def test_exposure_config1(U):
     ro = synth.rollout(0, 4, 8, 256)
-    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    omega = oracle_omega(ro)
     rms = _rms_for(ro, U, 1)
     E, sw = G.unit_exposure(omega, ro.mask, rms)
     oE, osw = oracle.unit_exposure(omega, ro.mask, rms)
@@ -140,7 +146,7 @@ def test_exposure_config1(U):
 def test_exposure_masked_microbatch_and_row_shift():
     """Microbatch of 4 responses x 4096 slots with padding; both row conventions."""
     ro = synth.rollout(0, 1, 4, 4096, rewards="uniform", lengths="uniform", mask_first_column=True)
-    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    omega = oracle_omega(ro)
     rms = _rms_for(ro, 5, 2)
     rms[:, ro.mask.reshape(-1) == 0] = 1e9          # padded rows must not contribute
     for shift in (0, 1):
@@ -157,7 +163,7 @@ def test_exposure_masked_microbatch_and_row_shift():
 
 def test_exposure_degenerate_cases():
     ro = synth.rollout(5, 2, 4, 64)
-    omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
+    omega = oracle_omega(ro)
     rms = _rms_for(ro, 3, 3)
     E, sw = G.unit_exposure(np.zeros_like(omega), ro.mask, rms)
     assert np.all(E == 0) and sw == 0                       # all coefficients zero
@@ -174,7 +180,8 @@ def test_exposure_degenerate_cases():
 
 
 def test_exposure_from_fused_token_rms():
-    """End of the chain: token RMS written by hilore_compress feeds hilore_unit_exposure."""
+    """End of the chain on the device (coefficients and token RMS as the kernels wrote them feed
+    hilore_unit_exposure) against the oracle's own chain."""
     ro = synth.rollout(0, 4, 8, 256)
     omega = G.grpo_coeffs(ro, N_norm=ro.n_valid)["omega"]
     rng = np.random.default_rng(0)
@@ -182,7 +189,7 @@ def test_exposure_from_fused_token_rms():
     rms = np.stack([G.compress(x, api.FMT_E4M3FN_BLK)[2] for x in units])
     E, _ = G.unit_exposure(omega, ro.mask, rms)
     o_rms = np.stack([oracle.row_rms(x) for x in units])
-    oE, _ = oracle.unit_exposure(omega, ro.mask, o_rms)
+    oE, _ = oracle.unit_exposure(oracle_omega(ro), ro.mask, o_rms)
     assert G.rel_err(E, oE).max() <= RTOL
 
 
