@@ -31,10 +31,9 @@ WORKLOAD = "1.5B-shaped: 64 prompts x G=8 x 1024 tokens; microbatch of 8 respons
            "28 layers x (1536, 1536, 8960) bf16 units, all L, E4M3FN + fp32 scale per 64"
 P, G_, T, MB_RESP, LAYERS, MODEL = 64, 8, 1024, 8, 28, "1.5B"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) per algorithmic byte of the two codec kernels, from the ncu captures
-# summarised in profiles/codec_kernels_bench_1p5B_and_unit8192x8960.md (section 4: one 7B-shaped unit
-# [16384, 18944], 950.5 MB algorithmic, five times the L2; traffic grows in proportion to the elements
-# processed).  Reads match the algorithmic reads (compress 1.02x, recover 1.00x); a few percent of the written
+# DRAM bytes (read + write) per algorithmic byte of the two codec kernels, from ncu captures of one 7B-shaped
+# unit [16384, 18944] (950.5 MB algorithmic, five times the L2; summarised under profiles/; traffic grows in
+# proportion to the elements processed).  Reads match the algorithmic reads (compress 1.02x, recover 1.00x); a few percent of the written
 # bytes are still dirty in L2 when such a single-unit kernel ends.
 DRAM_PER_ALGORITHMIC = {"compress": (633.987072 + 313.676288) / 950.5,
                         "recover": (330.265088 + 562.327808) / 950.4}
