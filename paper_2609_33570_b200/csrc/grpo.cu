@@ -390,86 +390,97 @@ struct ExpArgs {
     int ntiles;
     const int32_t *cu; // packed layout: sequence boundaries (else nullptr: rows of T slots)
     int n_seq;
+    int steps;         // pieces of kExpTile slots per CTA
 };
 
+// A CTA covers `steps` consecutive pieces of kExpTile slots for kExpUnits units: every thread accumulates its
+// slots of all pieces in registers (fp32) and the warp / CTA reduction runs once per CTA, so that the reduction
+// no longer costs more than the loads on large token grids.
 template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __grid_constant__ ExpArgs a)
 {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int tile = blockIdx.x;
     const int u0 = blockIdx.y * kExpUnits, nu = min(kExpUnits, a.U - u0);
-    float wabs[4];   // |omega| at valid slots, else 0
-    bool mk[4];      // slot is in T_b
-    bool has[4];     // ... and its activation row exists (t - row_shift >= 0)
-    int64_t slot[4];
-    if (VEC) {
-        const int64_t k = (int64_t)tile * kExpTile + (int64_t)tid * 4;
+    __shared__ double sm[kExpThreads / 32][2 * (kExpUnits + 1)];
+    // per-thread partials in fp32 (four terms per piece), warp tree in fp32, across warps and tiles in fp64
+    float acc[2 * (kExpUnits + 1)];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) slot[i] = k + i;
-        if (k < a.n_tok) { // n_tok % 4 == 0: a group is valid as a whole
-            const float4 w = *reinterpret_cast<const float4 *>(a.omega + k);
-            const uint32_t m = *reinterpret_cast<const unsigned int *>(a.mask + k);
-            const float wv[4] = {w.x, w.y, w.z, w.w};
+    for (int q = 0; q < 2 * (kExpUnits + 1); ++q) acc[q] = 0.0f;
+    for (int st = 0; st < a.steps; ++st) {
+        const int64_t piece = (int64_t)tile * a.steps + st;
+        if (piece * kExpTile >= a.n_tok)
+            break;
+        float wabs[4];   // |omega| at valid slots, else 0
+        bool mk[4];      // slot is in T_b
+        bool has[4];     // ... and its activation row exists (t - row_shift >= 0)
+        int64_t slot[4];
+        if (VEC) {
+            const int64_t k = piece * kExpTile + (int64_t)tid * 4;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                mk[i] = ((m >> (8 * i)) & 0xFFu) != 0;
-                has[i] = mk[i];
-                wabs[i] = mk[i] ? fabsf(wv[i]) : 0.0f;
+            for (int i = 0; i < 4; ++i) slot[i] = k + i;
+            if (k < a.n_tok) { // n_tok % 4 == 0: a group is valid as a whole
+                const float4 w = *reinterpret_cast<const float4 *>(a.omega + k);
+                const uint32_t m = *reinterpret_cast<const unsigned int *>(a.mask + k);
+                const float wv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    mk[i] = ((m >> (8 * i)) & 0xFFu) != 0;
+                    has[i] = mk[i];
+                    wabs[i] = mk[i] ? fabsf(wv[i]) : 0.0f;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    mk[i] = false;
+                    has[i] = false;
+                    wabs[i] = 0.0f;
+                }
             }
         } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
+                const int64_t k = piece * kExpTile + i * kExpThreads + tid;
+                slot[i] = k;
                 mk[i] = false;
                 has[i] = false;
                 wabs[i] = 0.0f;
-            }
-        }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int64_t k = (int64_t)tile * kExpTile + i * kExpThreads + tid;
-            slot[i] = k;
-            mk[i] = false;
-            has[i] = false;
-            wabs[i] = 0.0f;
-            if (k < a.n_tok && a.mask[k] != 0) {
-                mk[i] = true;
-                wabs[i] = fabsf(a.omega[k]);
-                // a slot whose source row lies before the start of its response has no activation term
-                if (a.row_shift == 0) has[i] = true;
-                else if (a.cu) has[i] = k - (int64_t)__ldg(a.cu + owner_sequence(a.cu, a.n_seq, k)) >= a.row_shift;
-                else has[i] = (k % a.T) >= a.row_shift;
-            }
-        }
-    }
-    __shared__ double sm[kExpThreads / 32][2 * (kExpUnits + 1)];
-    // per-thread partials in fp32 (four terms), warp tree in fp32, across warps and tiles in fp64
-    float acc[2 * (kExpUnits + 1)];
-    acc[2 * kExpUnits] = (wabs[0] + wabs[1]) + (wabs[2] + wabs[3]);
-    acc[2 * kExpUnits + 1] = (float)((int)mk[0] + (int)mk[1] + (int)mk[2] + (int)mk[3]);
-#pragma unroll
-    for (int j = 0; j < kExpUnits; ++j) {
-        float s1 = 0.0f, s2 = 0.0f;
-        if (j < nu) {
-            const float *ar = a.row_rms + (int64_t)(u0 + j) * a.rms_ld;
-            float av[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-            if (VEC) {
-                if (slot[0] < a.n_tok) {
-                    const float4 t = *reinterpret_cast<const float4 *>(ar + slot[0]);
-                    av[0] = t.x; av[1] = t.y; av[2] = t.z; av[3] = t.w;
+                if (k < a.n_tok && a.mask[k] != 0) {
+                    mk[i] = true;
+                    wabs[i] = fabsf(a.omega[k]);
+                    // a slot whose source row lies before the start of its response has no activation term
+                    if (a.row_shift == 0) has[i] = true;
+                    else if (a.cu) has[i] = k - (int64_t)__ldg(a.cu + owner_sequence(a.cu, a.n_seq, k)) >= a.row_shift;
+                    else has[i] = (k % a.T) >= a.row_shift;
                 }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (has[i]) av[i] = ar[slot[i] - a.row_shift];
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                s1 += has[i] ? av[i] : 0.0f;
-                s2 = fmaf(wabs[i], has[i] ? av[i] : 0.0f, s2);
             }
         }
-        acc[2 * j] = s1;
-        acc[2 * j + 1] = s2;
+        acc[2 * kExpUnits] += (wabs[0] + wabs[1]) + (wabs[2] + wabs[3]);
+        acc[2 * kExpUnits + 1] += (float)((int)mk[0] + (int)mk[1] + (int)mk[2] + (int)mk[3]);
+#pragma unroll
+        for (int j = 0; j < kExpUnits; ++j) {
+            float s1 = 0.0f, s2 = 0.0f;
+            if (j < nu) {
+                const float *ar = a.row_rms + (int64_t)(u0 + j) * a.rms_ld;
+                float av[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                if (VEC) {
+                    if (slot[0] < a.n_tok) {
+                        const float4 t = *reinterpret_cast<const float4 *>(ar + slot[0]);
+                        av[0] = t.x; av[1] = t.y; av[2] = t.z; av[3] = t.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (has[i]) av[i] = ar[slot[i] - a.row_shift];
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    s1 += has[i] ? av[i] : 0.0f;
+                    s2 = fmaf(wabs[i], has[i] ? av[i] : 0.0f, s2);
+                }
+            }
+            acc[2 * j] += s1;
+            acc[2 * j + 1] += s2;
+        }
     }
 #pragma unroll
     for (int q = 0; q < 2 * (kExpUnits + 1); ++q) {
@@ -649,9 +660,15 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
         return HILORE_ALIGN;
     if (workspace_bytes < hilore_workspace_bytes(U, n_tok))
         return HILORE_WORKSPACE;
-    const int64_t ntiles64 = (n_tok + kExpTile - 1) / kExpTile;
-    if (ntiles64 > 0x7FFFFFFF || (U + kExpUnits - 1) / kExpUnits > 65535)
+    const int64_t pieces = (n_tok + kExpTile - 1) / kExpTile;
+    const int64_t groups = (U + kExpUnits - 1) / kExpUnits;
+    if (pieces > 0x7FFFFFFF || groups > 65535)
         return HILORE_SHAPE;
+    // pieces per CTA: as many (up to 8) as still leave two full waves of CTAs
+    int steps = 1;
+    while (steps < 8 && (pieces / (2 * steps)) * groups >= 2ll * sm_count() * 8)
+        steps *= 2;
+    const int64_t ntiles64 = (pieces + steps - 1) / steps;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ExpArgs a{};
     a.omega = omega;
@@ -667,6 +684,7 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     a.ntiles = (int)ntiles64;
     a.cu = cu;
     a.n_seq = (int)n_seq;
+    a.steps = steps;
     if (a.ntiles > 0) {
         const dim3 grid((unsigned)a.ntiles, (unsigned)((U + kExpUnits - 1) / kExpUnits));
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&

@@ -91,6 +91,25 @@ def relerr_point(rows, cols, fmt, reps):
             "gbs": 2 * rows * cols / t / 1e6, "e": e.item()}
 
 
+def exposure_point(log2_tok, U, reps):
+    """hilore_unit_exposure over n_tok tokens and U units: n_tok * (5 + 4 U) bytes."""
+    n_tok = 1 << log2_tok
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    omega = torch.randn(n_tok, generator=gen, device="cuda") * 1e-5
+    mask = (torch.rand(n_tok, generator=gen, device="cuda") < 0.8).to(torch.uint8)
+    pool = max(1, min(4, -(-3 * L2_BYTES // (n_tok * 4 * U))))
+    rms = [torch.rand((U, n_tok), generator=gen, device="cuda") + 0.5 for _ in range(pool)]
+    out = torch.zeros(U, device="cuda")
+    nws = api.hilore_workspace_bytes(U, n_tok)
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    fns = [lambda i=i: api.hilore_unit_exposure(omega, mask, 1, n_tok, rms[i], U, n_tok, 0, 1e-8, out, None, ws, nws)
+           for i in range(pool)]
+    t = _time(fns, reps)
+    return {"kernel": "unit_exposure", "n_tok": n_tok, "U": U, "pool": pool, "us": t * 1e3,
+            "gbs": n_tok * (5 + 4 * U) / t / 1e6}
+
+
 def coeffs_packed_point(log2_tokens, reps, G=8, mean_len=2048):
     """The coefficient kernel on the packed layout: sequences of U{mean_len/2 .. 3 mean_len/2} tokens back to back."""
     import numpy as np
@@ -194,6 +213,8 @@ def main():
             print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
         for fmt in a.fmts:
             print(json.dumps(relerr_point(65536, 8960, fmt, a.reps)), flush=True)
+        for ls, U in ((13, 84), (17, 84), (20, 84), (24, 12)):
+            print(json.dumps(exposure_point(ls, U, a.reps)), flush=True)
         for ls in (15, 20, 24, 27):
             print(json.dumps(coeffs_packed_point(ls, a.reps)), flush=True)
         for ls in (20, 24, 27):
