@@ -156,3 +156,30 @@ def test_error_statistic_of_gpu_roundtrip_matches_oracle():
     o_rec = oracle.recover(o_codes, None, 0, 0)
     assert np.array_equal(codes, o_codes) and np.array_equal(rec, o_rec)
     assert 0.02 < oracle.relative_error(x, o_rec) < 0.035
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_leading_dimensions_and_specials(seed):
+    """Random rows / widths / leading dimensions / formats with special values sprinkled in (zeros, tiny and huge
+    magnitudes, Inf, NaN, whole blocks of one value): everything bit-exact against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    for _ in range(5):
+        rows = int(rng.integers(1, 700))
+        cols = 64 * int(rng.integers(1, 80))
+        pad = 16 * int(rng.integers(0, 4))
+        fmt = FMTS[int(rng.integers(0, 3))]
+        x = synth.activation_unit(rng, rows, cols)
+        n_special = int(rng.integers(0, 40))
+        specials = np.array([0x0000, 0x8000, 0x0001, 0x007F, 0x0080, 0x03E0, 0x03E1, 0x04DF, 0x04E0, 0x02FE, 0x03FE, 0x43E8, 0x43E9,
+                             0x7F7F, 0xFF7F, 0x7F80, 0xFF80, 0x7FC0, 0xFFC1, 0x3F80], np.uint16)
+        r_idx, c_idx = rng.integers(0, rows, n_special), rng.integers(0, cols, n_special)
+        x[r_idx, c_idx] = specials[rng.integers(0, len(specials), n_special)]
+        for _ in range(int(rng.integers(0, 4))):                      # whole blocks of one special value
+            r, b = int(rng.integers(0, rows)), int(rng.integers(0, cols // 64))
+            x[r, 64 * b:64 * b + 64] = specials[int(rng.integers(0, len(specials)))]
+        if pad:
+            wide = np.full((rows, cols + pad), 0x7FC0, np.uint16)      # NaN padding: must never be read
+            wide[:, :cols] = x
+            check_roundtrip(wide, fmt, cols=cols, ld_out=cols + 16 * int(rng.integers(0, 3)))
+        else:
+            check_roundtrip(x, fmt)
