@@ -206,3 +206,23 @@ def test_ratio_over_the_whole_exponent_range():
     near = (np.abs(r - hi) <= 4 * np.spacing(hi)) | (np.abs(r - lo) <= 4 * np.spacing(lo))
     assert np.array_equal(got["chi"][~near], chi[~near])
     assert G.rel_err(got["omega"][~near], w[~near]).max() <= RTOL
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_rollouts_and_microbatch_slices(seed):
+    """Random group sizes, lengths, rewards, clip radii, KL weights and microbatch slices against the oracle."""
+    rng = np.random.default_rng(500 + seed)
+    for _ in range(4):
+        Gs = int(rng.choice([1, 2, 4, 8, 16, 32, 48]))
+        P = int(rng.integers(1, 9))
+        T = 4 * int(rng.integers(1, 600))
+        ro = synth.rollout(int(rng.integers(0, 1 << 30)), P, Gs, T, rewards=str(rng.choice(["bernoulli", "uniform"])),
+                           lengths=str(rng.choice(["full", "uniform"])), min_len=1,
+                           equal_group_fraction=float(rng.choice([0.0, 0.5])))
+        ro.logp_old[:] = ro.logp_new + rng.normal(0, float(rng.choice([0.01, 0.1, 0.4])), ro.logp_new.shape).astype(np.float32)
+        beta = float(rng.choice([0.0, 1e-3, 0.3]))
+        clip = float(rng.choice([0.1, 0.2, 0.28]))
+        off = int(rng.integers(0, ro.n_resp))
+        n_rows = int(rng.integers(1, ro.n_resp - off + 1))
+        got = G.grpo_coeffs(ro, resp_offset=off, n_rows=n_rows, N_norm=ro.n_valid, clip_eps=clip, beta=beta)
+        check_coeffs(ro, got, resp_offset=off, beta=beta, clip_eps=clip)
