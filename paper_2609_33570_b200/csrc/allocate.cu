@@ -72,17 +72,16 @@ struct AllocArgs {
     double *totals;
 };
 
-constexpr int kAllocThreads = 512;
+constexpr int kAllocThreads = 1024;
 
 // The whole allocation in one cooperative launch: integer costs, the U layers of the DP (each a grid-stride
 // pass over the states, separated by grid-wide barriers), the terminal maximum and the backtracking.
 //   F_i(j,k) = max over available a with b <= j, r <= k of F_{i-1}(j-b, k-r) + tau_i(a); candidates in the
 //   order R, H, L, the first maximum wins.
-__global__ void __launch_bounds__(kAllocThreads) alloc_dp_kernel(const __grid_constant__ AllocArgs a)
+__global__ void __launch_bounds__(kAllocThreads, 2) alloc_dp_kernel(const __grid_constant__ AllocArgs a)
 {
     namespace cg = cooperative_groups;
     cg::grid_group grid = cg::this_grid();
-    __shared__ AllocUnit su;
     __shared__ Terminal sm[kAllocThreads];
     const int64_t S = (int64_t)a.KB * a.KD;
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, gsz = (int64_t)gridDim.x * blockDim.x;
@@ -94,36 +93,48 @@ __global__ void __launch_bounds__(kAllocThreads) alloc_dp_kernel(const __grid_co
     grid.sync();
 
     double *Fprev = a.F0, *Fcur = a.F1;
+    const int KD = a.KD;
+    // (j, k) of this thread's first state and the step between its states (no division in the loops)
+    const int j0 = (int)(gid / KD), k0 = (int)(gid - (int64_t)j0 * KD);
+    const int dj = (int)(gsz / KD), dk = (int)(gsz - (int64_t)dj * KD);
+    const double ninf = -INFINITY;
     for (int u = 0; u < a.U; ++u) {
-        if (threadIdx.x == 0)
-            su = a.units[u];
-        __syncthreads();
+        // Candidates in the order R, H, L; R always costs (0, 0) and adds 0, so it is the state itself.
+        // An unavailable action gets a cost no state can pay.
+        const AllocUnit un = a.units[u]; // the same 48 bytes for every thread: one broadcast load per layer
+        const int bH = un.b[HILORE_ACT_H] < 0 ? 0x3FFFFFFF : un.b[HILORE_ACT_H], rH = un.r[HILORE_ACT_H] < 0 ? 0 : un.r[HILORE_ACT_H];
+        const int bL = un.b[HILORE_ACT_L] < 0 ? 0x3FFFFFFF : un.b[HILORE_ACT_L], rL = un.r[HILORE_ACT_L] < 0 ? 0 : un.r[HILORE_ACT_L];
+        const int offH = bH < 0x3FFFFFFF ? bH * KD + rH : 0, offL = bL < 0x3FFFFFFF ? bL * KD + rL : 0;
+        const double tH = un.tau[HILORE_ACT_H], tL = un.tau[HILORE_ACT_L];
         uint8_t *pred = a.pred + (size_t)u * S;
-        // (j, k) of this thread's states, advanced incrementally (no division in the loop)
-        int j = (int)(gid / a.KD), k = (int)(gid - (int64_t)j * a.KD);
-        const int dj = (int)(gsz / a.KD), dk = (int)(gsz - (int64_t)dj * a.KD);
-        for (int64_t s = gid; s < S; s += gsz, j += dj, k += dk) {
-            if (k >= a.KD) {
-                k -= a.KD;
+        int j = j0, k = k0;
+        for (int s = (int)gid; s < (int)S; s += (int)gsz, j += dj, k += dk) {
+            if (k >= KD) {
+                k -= KD;
                 ++j;
             }
-            double best = -INFINITY;
-            uint32_t arg = 255;
-#pragma unroll
-            for (int c = 0; c < 3; ++c) {
-                const int b = su.b[c], r = su.r[c];
-                if (b < 0 || b > j || r > k)
-                    continue;
-                const double prev = Fprev[(int64_t)(j - b) * a.KD + (k - r)];
-                if (prev == -INFINITY)
-                    continue;
-                const double v = prev + su.tau[c];
-                if (arg == 255 || v > best) {
+            const bool canH = j >= bH && k >= rH, canL = j >= bL && k >= rL;
+            // the three reads are issued together
+            const double pR = Fprev[s];
+            const double pH = canH ? Fprev[s - offH] : ninf;
+            const double pL = canL ? Fprev[s - offL] : ninf;
+            double best = pR; // pR + 0.0 is pR for every value the table can hold
+            uint32_t arg = (pR == ninf) ? 255u : (uint32_t)HILORE_ACT_R;
+            if (pH != ninf) {
+                const double v = pH + tH;
+                if (arg == 255u || v > best) {
                     best = v;
-                    arg = c;
+                    arg = HILORE_ACT_H;
                 }
             }
-            Fcur[s] = best;
+            if (pL != ninf) {
+                const double v = pL + tL;
+                if (arg == 255u || v > best) {
+                    best = v;
+                    arg = HILORE_ACT_L;
+                }
+            }
+            Fcur[s] = (arg == 255u) ? ninf : best;
             pred[s] = (uint8_t)arg;
         }
         grid.sync();
