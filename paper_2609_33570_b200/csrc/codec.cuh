@@ -525,8 +525,8 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
                 bool careful = false;
                 process_pair<FMT, CODES, SUMS, true>(wa, wb, lane, qa, qb, s, ss, careful, tab);
                 if (CODES) {
-                    *reinterpret_cast<uint4 *>(cp) = qa;
-                    *reinterpret_cast<uint4 *>(cp + kCodecThreads * 16) = qb;
+                    __stcs(reinterpret_cast<uint4 *>(cp), qa);
+                    __stcs(reinterpret_cast<uint4 *>(cp + kCodecThreads * 16), qb);
                     if (FMT != HILORE_FMT_E4M3FN_RAW) {
                         if (q == 0) sp[0] = s;
                         if (q == 2) sp[kCodecThreads / 4] = s;
