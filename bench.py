@@ -148,7 +148,6 @@ class Workload:
         self.kappa = torch.from_numpy(kgen.uniform(0.5, 2.0, self.U).astype(np.float32)).to(device)
         self.ebar = torch.full((self.U,), 0.025, dtype=torch.float32, device=device)
         self.omega = torch.empty((MB_RESP, T), dtype=torch.float32, device=device)
-        self.adv = torch.empty(MB_RESP, dtype=torch.float32, device=device)
         self.ws_bytes = api.hilore_workspace_bytes(self.U, self.rows)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
         self.n_valid = ro.n_valid
@@ -158,7 +157,7 @@ class Workload:
         self.bytes_coeffs = coeff_bytes(self.rows)
         self.bytes_exposure = exposure_bytes(self.rows, self.U)
         self.bytes_step = self.bytes_compress + self.bytes_recover + self.bytes_coeffs + self.bytes_exposure
-        self.launches_per_step = 6
+        self.launches_per_step = 5   # capture, scores (2), decide, recover
 
     def step(self, mb: int, ev=None):
         """One microbatch: capture (compress all L candidates + token RMS), coefficients, exposure,
@@ -171,15 +170,11 @@ class Workload:
         api.hilore_plan_apply(self.units_dev, self.units_host, self.U, api.PHASE_CAPTURE, None, None, None, 0.0, 0.0,
                               self.avail, self.action, None, None, None)
         rec("compress", 1)
-        rec("coeffs", 0)
-        api.hilore_grpo_coeffs(self.rewards, self.n_resp, G_, mb * MB_RESP, MB_RESP, T, self.logp_new[sl],
-                               self.logp_old[sl], None, self.mask[sl], self.n_valid, None, 0.2, 0.0, 1e-6,
-                               self.adv, self.omega, None, None)
-        rec("coeffs", 1)
-        rec("exposure", 0)
-        api.hilore_unit_exposure(self.omega, self.mask[sl], MB_RESP, T, self.rms, self.U, self.rows, 0, 1e-8,
-                                 self.exposure, None, self.ws, self.ws_bytes)
-        rec("exposure", 1)
+        rec("scores", 0)   # coefficients and their reduction to exposure scores: one sweep (two launches)
+        api.hilore_coeffs_exposure(self.rewards, self.n_resp, G_, mb * MB_RESP, MB_RESP, T, self.logp_new[sl],
+                                   self.logp_old[sl], None, self.mask[sl], self.n_valid, None, 0.2, 0.0, 1e-6, self.rms,
+                                   self.U, self.rows, 0, 1e-8, self.omega, self.exposure, None, self.ws, self.ws_bytes)
+        rec("scores", 1)
         api.hilore_plan_apply(self.units_dev, self.units_host, self.U, api.PHASE_DECIDE, self.exposure, self.kappa,
                               self.ebar, inf, inf, self.avail, self.action, self.psi, self.recompute, self.retained)
         rec("recover", 0)
@@ -329,7 +324,7 @@ def main():
 
     for i in range(args.warmup):
         wl.step(i % wl.n_microbatches)
-    kinds = ("compress", "coeffs", "exposure", "recover")
+    kinds = ("compress", "scores", "recover")
     evs = [{k: (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for k in kinds}
            for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -421,8 +416,8 @@ def main():
         "kernels": {
             "compress": {"ms": kern_ms["compress"], "gbs": wl.bytes_compress / kern_ms["compress"] / 1e6},
             "recover": {"ms": kern_ms["recover"], "gbs": wl.bytes_recover / kern_ms["recover"] / 1e6},
-            "coeffs_microbatch": {"ms": kern_ms["coeffs"], "tokens_per_s": wl.rows / kern_ms["coeffs"] * 1e3},
-            "exposure": {"ms": kern_ms["exposure"], "gbs": wl.bytes_exposure / kern_ms["exposure"] / 1e6},
+            "scores_microbatch": {"ms": kern_ms["scores"], "tokens_per_s": wl.rows / kern_ms["scores"] * 1e3,
+                                  "gbs": (wl.bytes_coeffs + wl.bytes_exposure) / kern_ms["scores"] / 1e6},
             "coeffs_2p24": sweep,
             "allocate_dp_u84_n1024": {"ms": alloc["us"] / 1e3, "state_updates_per_s": alloc["state_updates_per_s"]},
         },

@@ -111,6 +111,22 @@ int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, in
                        float *omega, float *ratio, uint8_t *clip_mask, void *stream);
 
 /*
+ * hilore_grpo_coeffs followed by hilore_unit_exposure as ONE sweep (Algorithm 1, "coefficients" and "exposure"
+ * lines; Eqs. "update-coefficient", "mlp-weighted-exposure"): the coefficients are computed inside the exposure
+ * reduction instead of being written and read back, which saves a launch and the round trip of omega when the
+ * microbatch is small enough for the call to be launch-bound (n_rows * T <= 2^18 slots and at most 62 responses
+ * per 1024 slots; other shapes run the two passes in turn inside this call).  Results are bit for bit those of
+ * the two calls: omega [n_rows, T] (REQUIRED here, it is written either way), exposure [U], sum_abs_omega (opt).
+ * Arguments, status codes and workspace as in the two calls; adv_out, ratio and clip_mask are not produced.
+ */
+int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset, int64_t n_rows,
+                           int64_t T, const float *logp_new, const float *logp_old, const float *logp_ref,
+                           const uint8_t *mask, int64_t N_norm, const int64_t *N_norm_dev, float clip_eps, float beta,
+                           float adv_eps, const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                           float eps_alpha, float *omega, float *exposure, float *sum_abs_omega, void *workspace,
+                           size_t workspace_bytes, void *stream);
+
+/*
  * The coefficient and exposure passes on the packed (padding-removed) layout of the paper's DSR-sub execution
  * setting (Table "execution-configurations": "padding removal").  The sequences of a microbatch -- prompt
  * followed by the generated response, no padding slots -- lie back to back: sequence i (response

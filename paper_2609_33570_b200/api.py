@@ -27,7 +27,8 @@ EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "h
            "hilore_allocate", "hilore_allocate_workspace_bytes", "hilore_risk_budget",
            "hilore_relative_error", "hilore_relative_error_workspace_bytes", "hilore_fit_kappa",
            "hilore_grpo_coeffs_variant", "hilore_omega_diagnostics", "hilore_omega_diagnostics_workspace_bytes",
-           "hilore_grpo_coeffs_packed", "hilore_unit_exposure_packed", "hilore_codec_relative_error")
+           "hilore_grpo_coeffs_packed", "hilore_unit_exposure_packed", "hilore_codec_relative_error",
+           "hilore_coeffs_exposure")
 
 
 class HiloreUnit(C.Structure):
@@ -87,6 +88,8 @@ def lib() -> C.CDLL:
         _lib.hilore_grpo_coeffs_packed.argtypes = [vp, i64, i32, i64, i64, vp, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32,
                                                    vp, vp, vp, vp, vp]
         _lib.hilore_unit_exposure_packed.argtypes = [vp, vp, i64, vp, i64, vp, i32, i64, i32, f32, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_coeffs_exposure.argtypes = [vp, i64, i32, i64, i64, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32, vp, i32, i64,
+                                                i32, f32, vp, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_codec_relative_error.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_omega_diagnostics.argtypes = [vp, vp, vp, vp, i64, i64, f32, vp, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_omega_diagnostics_workspace_bytes.restype = C.c_size_t
@@ -168,6 +171,16 @@ def hilore_unit_exposure_packed(omega, mask, n_tok, cu_seqlens, n_seq, row_rms, 
                                            rms_ld, row_shift, eps_alpha, _ptr(exposure), _ptr(sum_abs_omega),
                                            _ptr(workspace), workspace_bytes, _stream(stream))
     return _check(st, "hilore_unit_exposure_packed", check)
+
+
+def hilore_coeffs_exposure(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask, N_norm,
+                           N_norm_dev, clip_eps, beta, adv_eps, row_rms, U, rms_ld, row_shift, eps_alpha, omega, exposure,
+                           sum_abs_omega, workspace, workspace_bytes, stream=None, check=True):
+    st = lib().hilore_coeffs_exposure(_ptr(rewards), n_resp_total, G, resp_offset, n_rows, T, _ptr(logp_new), _ptr(logp_old),
+                                      _ptr(logp_ref), _ptr(mask), N_norm, _ptr(N_norm_dev), clip_eps, beta, adv_eps,
+                                      _ptr(row_rms), U, rms_ld, row_shift, eps_alpha, _ptr(omega), _ptr(exposure),
+                                      _ptr(sum_abs_omega), _ptr(workspace), workspace_bytes, _stream(stream))
+    return _check(st, "hilore_coeffs_exposure", check)
 
 
 def hilore_codec_relative_error(x, rows, cols, ld, fmt, block, e_out, norms2, workspace, workspace_bytes, stream=None,

@@ -378,6 +378,19 @@ constexpr int kExpThreads = 256;
 constexpr int kExpTile = kExpThreads * 4; // slots per CTA
 constexpr int kExpUnits = 8;              // units per CTA (omega and mask are read once for all of them)
 
+// Inputs of the coefficient pass when it is fused into the exposure reduction (hilore_coeffs_exposure).
+constexpr int kFusedRows = 64; // responses one CTA's slots may span
+struct FusedCoeff {
+    const float *rewards;
+    int G;
+    int64_t resp_offset;
+    const float *logp_new, *logp_old, *logp_ref;
+    int64_t N_norm;
+    const long long *N_norm_dev;
+    float clip_eps, beta, adv_eps;
+    float *omega_out;
+};
+
 struct ExpArgs {
     const float *omega;
     const uint8_t *mask;
@@ -391,17 +404,54 @@ struct ExpArgs {
     const int32_t *cu; // packed layout: sequence boundaries (else nullptr: rows of T slots)
     int n_seq;
     int steps;         // pieces of kExpTile slots per CTA
+    FusedCoeff f;      // used by the fused kernel only
 };
 
 // A CTA covers `steps` consecutive pieces of kExpTile slots for kExpUnits units: every thread accumulates its
 // slots of all pieces in registers (fp32) and the warp / CTA reduction runs once per CTA, so that the reduction
 // no longer costs more than the loads on large token grids.
-template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __grid_constant__ ExpArgs a)
+// One coefficient, exactly as grpo_coeffs_kernel computes it (same expressions, same rounding).
+__device__ __forceinline__ float fused_omega(float s, float o, float rf, bool m, float A, float coef, float kl, float hi, float lo)
+{
+    const float r = exp_ratio(s - o);
+    const bool c = (A >= 0.0f) ? (r <= hi) : (r >= lo);
+    float v = (m && c) ? coef * r : 0.0f;
+    if (kl != 0.0f && m)
+        v += kl * (-expm1f(rf - s));
+    return v;
+}
+
+// FUSED: omega is not read but computed here from the log-probabilities (and written once, by the CTAs of the
+// first unit group): the coefficient pass and its reduction to exposure scores in one sweep.
+template <bool VEC, bool FUSED = false>
+__global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __grid_constant__ ExpArgs a)
 {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int tile = blockIdx.x;
     const int u0 = blockIdx.y * kExpUnits, nu = min(kExpUnits, a.U - u0);
     __shared__ double sm[kExpThreads / 32][2 * (kExpUnits + 1)];
+    __shared__ float s_A[FUSED ? kFusedRows : 1], s_coef[FUSED ? kFusedRows : 1];
+    int64_t row_lo = 0;
+    float f_kl = 0.0f, f_hi = 0.0f, f_lo = 0.0f;
+    if (FUSED) { // the per-response scalars of the responses this CTA's slots belong to
+        const int64_t slot_lo = (int64_t)tile * a.steps * kExpTile;
+        const int64_t slot_hi = min(a.n_tok, slot_lo + (int64_t)a.steps * kExpTile);
+        row_lo = slot_lo / a.T;
+        const int nrows = (int)((slot_hi - 1) / a.T - row_lo) + 1;
+        const long long N = a.f.N_norm_dev ? *a.f.N_norm_dev : (long long)a.f.N_norm;
+        const double invN = N > 0 ? 1.0 / (double)N : 0.0;
+        for (int r = wid; r < nrows; r += kExpThreads / 32) {
+            const float A = group_advantage(a.f.rewards, a.f.resp_offset + row_lo + r, a.f.G, a.f.adv_eps, lane);
+            if (lane == 0) {
+                s_A[r] = A;
+                s_coef[r] = (float)(-(double)A * invN);
+            }
+        }
+        f_kl = (float)((double)a.f.beta * invN);
+        f_hi = 1.0f + a.f.clip_eps;
+        f_lo = 1.0f - a.f.clip_eps;
+        __syncthreads();
+    }
     // per-thread partials in fp32 (four terms per piece), warp tree in fp32, across warps and tiles in fp64
     float acc[2 * (kExpUnits + 1)];
 #pragma unroll
@@ -419,9 +469,25 @@ template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_part
 #pragma unroll
             for (int i = 0; i < 4; ++i) slot[i] = k + i;
             if (k < a.n_tok) { // n_tok % 4 == 0: a group is valid as a whole
-                const float4 w = *reinterpret_cast<const float4 *>(a.omega + k);
                 const uint32_t m = *reinterpret_cast<const unsigned int *>(a.mask + k);
-                const float wv[4] = {w.x, w.y, w.z, w.w};
+                float wv[4];
+                if (FUSED) { // T % 4 == 0: the four slots belong to one response
+                    const float4 sn = *reinterpret_cast<const float4 *>(a.f.logp_new + k);
+                    const float4 so = *reinterpret_cast<const float4 *>(a.f.logp_old + k);
+                    float4 sr = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (f_kl != 0.0f) sr = *reinterpret_cast<const float4 *>(a.f.logp_ref + k);
+                    const int ri = (int)(k / a.T - row_lo);
+                    const float A = s_A[ri], coef = s_coef[ri];
+                    wv[0] = fused_omega(sn.x, so.x, sr.x, (m & 0xFFu) != 0, A, coef, f_kl, f_hi, f_lo);
+                    wv[1] = fused_omega(sn.y, so.y, sr.y, (m & 0xFF00u) != 0, A, coef, f_kl, f_hi, f_lo);
+                    wv[2] = fused_omega(sn.z, so.z, sr.z, (m & 0xFF0000u) != 0, A, coef, f_kl, f_hi, f_lo);
+                    wv[3] = fused_omega(sn.w, so.w, sr.w, (m & 0xFF000000u) != 0, A, coef, f_kl, f_hi, f_lo);
+                    if (a.f.omega_out && blockIdx.y == 0)
+                        *reinterpret_cast<float4 *>(a.f.omega_out + k) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+                } else {
+                    const float4 w = *reinterpret_cast<const float4 *>(a.omega + k);
+                    wv[0] = w.x; wv[1] = w.y; wv[2] = w.z; wv[3] = w.w;
+                }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     mk[i] = ((m >> (8 * i)) & 0xFFu) != 0;
@@ -444,9 +510,16 @@ template <bool VEC> __global__ void __launch_bounds__(kExpThreads) exposure_part
                 mk[i] = false;
                 has[i] = false;
                 wabs[i] = 0.0f;
+                if (FUSED && k < a.n_tok) { // every slot gets its coefficient, masked ones a zero
+                    const int ri = (int)(k / a.T - row_lo);
+                    const float w = fused_omega(a.f.logp_new[k], a.f.logp_old[k], f_kl != 0.0f ? a.f.logp_ref[k] : 0.0f,
+                                                a.mask[k] != 0, s_A[ri], s_coef[ri], f_kl, f_hi, f_lo);
+                    if (a.f.omega_out && blockIdx.y == 0) a.f.omega_out[k] = w;
+                    wabs[i] = fabsf(w);
+                }
                 if (k < a.n_tok && a.mask[k] != 0) {
                     mk[i] = true;
-                    wabs[i] = fabsf(a.omega[k]);
+                    if (!FUSED) wabs[i] = fabsf(a.omega[k]);
                     // a slot whose source row lies before the start of its response has no activation term
                     if (a.row_shift == 0) has[i] = true;
                     else if (a.cu) has[i] = k - (int64_t)__ldg(a.cu + owner_sequence(a.cu, a.n_seq, k)) >= a.row_shift;
@@ -640,10 +713,12 @@ extern "C" size_t hilore_workspace_bytes(int32_t U, int64_t n_tok)
     return (size_t)(U + 1) * (size_t)(ntiles > 0 ? ntiles : 1) * 2 * sizeof(double);
 }
 
+// fused: compute omega inside the reduction (hilore_coeffs_exposure); *fused_done tells the caller whether that was
+// possible for this shape (otherwise nothing has been launched and the caller runs the two passes in turn).
 static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T, int64_t n_tok,
                            const int32_t *cu, int64_t n_seq, const float *row_rms, int32_t U, int64_t rms_ld,
                            int32_t row_shift, float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
-                           size_t workspace_bytes, void *stream)
+                           size_t workspace_bytes, void *stream, const FusedCoeff *fused = nullptr, bool *fused_done = nullptr)
 {
     if (n_rows < 0 || T < 0 || n_tok < 0 || U < 0 || row_shift < 0 || row_shift > 1)
         return HILORE_INVALID_ARG;
@@ -669,8 +744,16 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     while (steps < 8 && (pieces / (2 * steps)) * groups >= 2ll * sm_count() * 8)
         steps *= 2;
     const int64_t ntiles64 = (pieces + steps - 1) / steps;
+    if (fused) { // a CTA keeps the scalars of the responses its slots span in shared memory; recomputing omega in
+                 // every unit group only pays while the call is launch-bound
+        const bool ok = T > 0 && ((int64_t)steps * kExpTile) / T + 2 <= kFusedRows && n_tok <= (1ll << 18);
+        *fused_done = ok;
+        if (!ok)
+            return HILORE_OK;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ExpArgs a{};
+    if (fused) a.f = *fused;
     a.omega = omega;
     a.mask = mask;
     a.n_rows = n_rows;
@@ -689,7 +772,12 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
         const dim3 grid((unsigned)a.ntiles, (unsigned)((U + kExpUnits - 1) / kExpUnits));
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
                          aligned(mask, 4) && aligned(row_rms, 16);
-        if (vec) exposure_partial_kernel<true><<<grid, kExpThreads, 0, st>>>(a);
+        if (fused) {
+            const bool fvec = vec && aligned(fused->logp_new, 16) && aligned(fused->logp_old, 16) && aligned(fused->logp_ref, 16) &&
+                              aligned(fused->omega_out, 16);
+            if (fvec) exposure_partial_kernel<true, true><<<grid, kExpThreads, 0, st>>>(a);
+            else exposure_partial_kernel<false, true><<<grid, kExpThreads, 0, st>>>(a);
+        } else if (vec) exposure_partial_kernel<true><<<grid, kExpThreads, 0, st>>>(a);
         else exposure_partial_kernel<false><<<grid, kExpThreads, 0, st>>>(a);
         if (cudaGetLastError() != cudaSuccess)
             return HILORE_CUDA;
@@ -707,6 +795,57 @@ extern "C" int hilore_unit_exposure(const float *omega, const uint8_t *mask, int
         return HILORE_INVALID_ARG;
     return launch_exposure(omega, mask, n_rows, T, n_rows * T, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha,
                            exposure, sum_abs_omega, workspace, workspace_bytes, stream);
+}
+
+extern "C" int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset, int64_t n_rows,
+                                      int64_t T, const float *logp_new, const float *logp_old, const float *logp_ref,
+                                      const uint8_t *mask, int64_t N_norm, const int64_t *N_norm_dev, float clip_eps, float beta,
+                                      float adv_eps, const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                      float eps_alpha, float *omega, float *exposure, float *sum_abs_omega, void *workspace,
+                                      size_t workspace_bytes, void *stream)
+{
+    // the argument rules of the two calls it stands for
+    if (rewards == nullptr || n_resp_total < 0 || G <= 0 || resp_offset < 0 || n_rows < 0 || T < 0 || U < 0)
+        return HILORE_INVALID_ARG;
+    if (n_resp_total % G != 0 || resp_offset + n_rows > n_resp_total || T % 4 != 0)
+        return HILORE_SHAPE;
+    if (beta != 0.0f && logp_ref == nullptr)
+        return HILORE_INVALID_ARG;
+    if (N_norm_dev == nullptr && N_norm <= 0)
+        return HILORE_ZERO_NORM;
+    const int64_t n_tok = n_rows * T;
+    if (n_tok > 0 && (logp_new == nullptr || logp_old == nullptr || mask == nullptr || omega == nullptr))
+        return HILORE_INVALID_ARG;
+    if (!aligned(logp_new, 16) || !aligned(logp_old, 16) || !aligned(logp_ref, 16) || !aligned(omega, 16) || !aligned(mask, 4) ||
+        !aligned(rewards, 4) || !aligned(N_norm_dev, 8))
+        return HILORE_ALIGN;
+    FusedCoeff f{};
+    f.rewards = rewards;
+    f.G = G;
+    f.resp_offset = resp_offset;
+    f.logp_new = logp_new;
+    f.logp_old = logp_old;
+    f.logp_ref = beta != 0.0f ? logp_ref : nullptr;
+    f.N_norm = N_norm;
+    f.N_norm_dev = reinterpret_cast<const long long *>(N_norm_dev);
+    f.clip_eps = clip_eps;
+    f.beta = beta;
+    f.adv_eps = adv_eps;
+    f.omega_out = omega;
+    bool fused_done = false;
+    if (U > 0 && n_tok > 0) {
+        const int st = launch_exposure(omega, mask, n_rows, T, n_tok, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha,
+                                       exposure, sum_abs_omega, workspace, workspace_bytes, stream, &f, &fused_done);
+        if (st != HILORE_OK || fused_done)
+            return st;
+    }
+    // shapes the fused kernel does not take (and U = 0): the two passes one after the other
+    const int st = launch_coeffs(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask, N_norm,
+                                 N_norm_dev, clip_eps, beta, adv_eps, 0, nullptr, omega, nullptr, nullptr, stream);
+    if (st != HILORE_OK)
+        return st;
+    return launch_exposure(omega, mask, n_rows, T, n_tok, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha, exposure,
+                           sum_abs_omega, workspace, workspace_bytes, stream);
 }
 
 extern "C" int hilore_unit_exposure_packed(const float *omega, const uint8_t *mask, int64_t n_tok,

@@ -21,7 +21,7 @@ def test_bench_line_has_the_contract_keys():
                 "vs_baseline", "dtype", "data", "config", "gpu_launches", "clocks", "roofline", "e2e"):
         assert key in d, key
     assert d["steps"] == 4 and d["warmup"] == 3 and d["n_gpus"] == 1 and d["vs_baseline"] is None
-    assert d["gpu_launches"] == 6 * 4 and "workload" in d["config"] and "model" not in d["config"]
+    assert d["gpu_launches"] == 5 * 4 and "workload" in d["config"] and "model" not in d["config"]
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert 0.3 < r["frac"] < 1.2 and r["traffic"] is not None

@@ -1,0 +1,69 @@
+"""hilore_coeffs_exposure (coefficients computed inside the exposure reduction): bit for bit the results of
+hilore_grpo_coeffs followed by hilore_unit_exposure, and within 1e-5 of the oracle's own chain."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_33570_b200 import api, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def fused(ro, rms, sl, beta=0.0, row_shift=0, N=None):
+    n_rows, T = sl.stop - sl.start, ro.T
+    U, ld = rms.shape
+    nws = api.hilore_workspace_bytes(U, n_rows * T)
+    ws, omega, E, sw = G.Guarded(nws), G.Guarded(n_rows * T * 4), G.Guarded(U * 4), G.Guarded(4)
+    api.hilore_coeffs_exposure(G.dev(ro.rewards), ro.n_resp, ro.G, sl.start, n_rows, T, G.dev(ro.logp_new[sl]), G.dev(ro.logp_old[sl]),
+                               G.dev(ro.logp_ref[sl]) if beta else None, G.dev(ro.mask[sl]), ro.n_valid if N is None else N, None,
+                               0.2, beta, 1e-6, G.dev(rms), U, ld, row_shift, 1e-8, omega.ptr(), E.ptr(), sw.ptr(), ws.ptr(), nws)
+    ws.numpy(np.uint8, (nws,))
+    return omega.numpy(np.float32, (n_rows, T)), E.numpy(np.float32, (U,)), float(sw.numpy(np.float32, (1,))[0])
+
+
+@pytest.mark.parametrize("P,G_,T,U,lengths,beta,row_shift", [
+    (4, 8, 256, 2, "full", 0.0, 0),            # the tiny configuration
+    (1, 8, 1024, 84, "full", 0.0, 0),          # one microbatch of the 1.5B-shaped configuration
+    (2, 4, 4096, 5, "uniform", 1e-3, 0),       # padding, KL term
+    (3, 4, 52, 3, "uniform", 0.0, 1),          # short rows, many responses per tile, shifted rows
+    (16, 16, 2048, 9, "uniform", 0.0, 0),      # 2^19 slots: the call runs the two passes in turn
+    (64, 8, 16, 4, "full", 0.0, 0),            # 64 responses per 1024 slots: too many rows per tile for one sweep
+])
+def test_one_sweep_equals_the_two_calls_and_the_oracle(P, G_, T, U, lengths, beta, row_shift):
+    ro = synth.rollout(51, P, G_, T, lengths=lengths, min_len=2, rewards="uniform", mask_first_column=bool(row_shift))
+    ro.logp_old[:] = ro.logp_new + np.random.default_rng(3).normal(0, 0.1, ro.logp_new.shape).astype(np.float32)
+    sl = slice(0, ro.n_resp)
+    rms = np.random.default_rng(4).random((U, ro.n_resp * T + 8), dtype=np.float32) + np.float32(0.25)
+    omega, E, sw = fused(ro, rms, sl, beta=beta, row_shift=row_shift)
+    two = G.grpo_coeffs(ro, N_norm=ro.n_valid, beta=beta, extras=False)["omega"]
+    E2, sw2 = G.unit_exposure(two, ro.mask, rms, row_shift=row_shift)
+    assert omega.tobytes() == two.tobytes() and E.tobytes() == E2.tobytes() and sw == sw2
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, r, _ = oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, ro.logp_ref if beta else None, ro.mask, N_norm=ro.n_valid, beta=beta)
+    oE, osw = oracle.unit_exposure(w, ro.mask, rms, row_shift=row_shift)
+    assert G.rel_err(E, oE).max() <= 1e-5 and abs(sw - osw) <= 1e-5 * osw
+
+
+def test_microbatch_slice_of_a_rollout_batch():
+    ro = synth.rollout(52, 4, 16, 512, rewards="bernoulli", equal_group_fraction=0.25)
+    sl = slice(24, 40)                                        # straddles two prompt groups
+    rms = np.random.default_rng(5).random((7, 16 * 512), dtype=np.float32) + np.float32(0.5)
+    omega, E, _ = fused(ro, rms, sl)
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, _, _ = oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=ro.n_valid)
+    oE, _ = oracle.unit_exposure(w, ro.mask[sl], rms)
+    assert G.rel_err(omega, w).max() <= 1e-5 and G.rel_err(E, oE).max() <= 1e-5
+
+
+def test_argument_errors():
+    z = torch.zeros(64, device="cuda")
+    m = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    call = lambda **k: api.hilore_coeffs_exposure(z, k.get("n_resp", 4), k.get("G", 4), 0, 4, k.get("T", 16), z, z, None, m,
+                                                  k.get("N", 3), None, 0.2, k.get("beta", 0.0), 1e-6, z, 1, 64, 0, 1e-8,
+                                                  k.get("omega", z), z, None, ws, k.get("nws", 4096), check=False)
+    assert call() == api.OK
+    assert call(omega=None) == api.INVALID_ARG and call(N=0) == api.ZERO_NORM and call(beta=0.5) == api.INVALID_ARG
+    assert call(T=18) == api.SHAPE and call(n_resp=5) == api.SHAPE and call(nws=8) == api.WORKSPACE
