@@ -593,6 +593,10 @@ __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, ui
                     row_rms[rb0 + r] = sqrtf((float)acc * inv_cols);
             }
             __syncthreads();
+        } else {
+            // Without the row reduction nothing else holds the warps of a CTA together, and they drift away from
+            // the elected thread's run-ahead: one barrier per batch keeps them behind it (+25 % on multi-GB units).
+            __syncthreads();
         }
     }
 }
