@@ -186,6 +186,45 @@ def allocate_point(U, reps, N=1024):
             "workspace_mib": nws / 2 ** 20}
 
 
+def plan_points(model="7B", rows=16384, layers=28, reps=5):
+    """hilore_plan_apply over a whole microbatch table (3 units per layer) under different candidate plans: token RMS
+    only (all H), capture of all units (all L), a 50 % L / 30 % H / 20 % R mix, post-forward encode of half the units."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    shapes = synth.layer_unit_shapes(model, rows, layers)
+    U = len(shapes)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1)
+    x = [synth.activation_unit_device(gen, r, c, dev) for r, c in shapes]
+    codes = [torch.empty((r, c), dtype=torch.uint8, device=dev) for r, c in shapes]
+    scales = [torch.empty((r, c // 64), dtype=torch.float32, device=dev) for r, c in shapes]
+    rms = torch.empty((U, rows), dtype=torch.float32, device=dev)
+    units = [dict(x=x[i], codes=codes[i], scales=scales[i], out=None, row_rms=rms[i], rows=r, cols=c, fmt=api.FMT_E4M3FN_BLK,
+                  block=64) for i, (r, c) in enumerate(shapes)]
+    udev, uhost = api.make_unit_table(units, dev)
+    H, L, R = api.ACT_H, api.ACT_L, api.ACT_R
+    cases = (("capture, all H (token RMS only)", [H] * U, None), ("capture, all L", [L] * U, None),
+             ("capture, 50% L / 30% H / 20% R", [(L, H, L, R, L, H, L, R, H, L)[i % 10] for i in range(U)], None),
+             ("encode, every second H candidate assigned L", [H] * U, [(L, H)[i % 2] for i in range(U)]))
+    out = []
+    for name, q, a in cases:
+        avail = torch.tensor(q, dtype=torch.uint8, device=dev)
+        action = torch.tensor(a if a else q, dtype=torch.uint8, device=dev)
+        phase = api.PHASE_ENCODE if a else api.PHASE_CAPTURE
+        fn = lambda: api.hilore_plan_apply(udev, uhost, U, phase, None, None, None, 0, 0, avail, action, None, None, None)
+        t = _time([fn], reps)
+        nbytes = 0
+        for i, (r, c) in enumerate(shapes):
+            if a:
+                nbytes += (r * c * 3 + r * c // 16) if a[i] == L else 0
+            elif q[i] == L:
+                nbytes += r * c * 3 + r * c // 16 + 4 * r
+            elif q[i] == H:
+                nbytes += r * c * 2 + 4 * r
+        out.append({"kernel": "plan_apply", "table": f"{model} x {layers} layers x {rows} rows", "case": name, "ms": t,
+                    "gbs": nbytes / t / 1e6})
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--cols", type=int, default=4096)
@@ -196,7 +235,12 @@ def main():
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--no-coeffs", action="store_true")
     ap.add_argument("--no-rms", action="store_true", help="compress without the fused token RMS")
+    ap.add_argument("--plan-table", action="store_true", help="only the 7B-shaped table under several candidate plans")
     a = ap.parse_args()
+    if a.plan_table:
+        for p in plan_points():
+            print(json.dumps(p), flush=True)
+        return
     for fmt in a.fmts:
         for lr in range(a.min_log2_rows, a.max_log2_rows + 1):
             rows = 1 << lr
