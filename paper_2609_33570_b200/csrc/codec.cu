@@ -49,8 +49,8 @@ template <int FMT> __device__ __forceinline__ void recover_unit(const hilore_uni
                                                                 uint32_t &tile, int prefetch)
 {
     uint16_t *out = static_cast<uint16_t *>(u.out);
-    if (u.ld == u.cols)
-        recover_rows_bulk<FMT>(u.codes, u.scales, out, u.cols, r0, r1, sm_out, tile, prefetch);
+    if (u.ld == u.cols || u.cols >= 1024) // wide enough rows: bulk stores also with a leading dimension
+        recover_rows_bulk<FMT>(u.codes, u.scales, out, u.cols, u.ld, r0, r1, sm_out, tile, prefetch);
     else
         recover_rows<FMT>(u.codes, u.scales, out, u.cols, u.ld, r0, r1, prefetch);
 }

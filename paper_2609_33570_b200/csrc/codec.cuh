@@ -717,22 +717,22 @@ constexpr int kRecoverTileChunks = 2 * kCodecThreads;        // 512 chunks = 819
 constexpr int kRecoverTileBytes = kRecoverTileChunks * 32;   // 16 KB of bf16
 constexpr int kRecoverStageBytes = 2 * kRecoverTileBytes;    // two tiles in shared memory
 
-// Decode rows [r0, r1) of a contiguous unit (ld == cols).  The pass writes twice what it reads, and HBM
-// takes writes best in large contiguous bursts: each tile of 8192 reconstructed values is assembled in
+// Decode rows [r0, r1) of a unit (contiguous, or rows of at least 2 KB with a leading dimension).  The pass
+// writes twice what it reads, and HBM takes writes best in large contiguous bursts: each tile of 8192 reconstructed values is assembled in
 // shared memory and sent with one 16 KB bulk store while the threads work on the next tile (two buffers;
 // a buffer is refilled only after the store that read it has finished reading).
 // `tile` counts this CTA's tiles across calls, so the two buffers keep alternating from unit to unit.
 template <int FMT>
 __device__ __forceinline__ void recover_rows_bulk(const uint8_t *__restrict__ codes, const float *__restrict__ scales,
-                                                  uint16_t *__restrict__ out, int64_t cols, int64_t r0, int64_t r1,
-                                                  uint8_t *sm_out, uint32_t &tile, int prefetch)
+                                                  uint16_t *__restrict__ out, int64_t cols, int64_t ld, int64_t r0,
+                                                  int64_t r1, uint8_t *sm_out, uint32_t &tile, int prefetch)
 {
     const int tid = threadIdx.x;
     const int64_t nb = cols >> 6, cpr = cols >> 4;
     const int64_t n = (r1 - r0) * cpr; // chunks of this CTA's rows
     const uint8_t *cb_ = codes + r0 * cols;
     const float *sb = scales + r0 * nb;
-    uint8_t *ob = reinterpret_cast<uint8_t *>(out + r0 * cols);
+    uint8_t *ob = reinterpret_cast<uint8_t *>(out + r0 * ld);
     const int64_t ntiles = (n + kRecoverTileChunks - 1) / kRecoverTileChunks;
     if (tid == 0)
         for (int64_t k = 0; k < prefetch && k < ntiles; ++k)
@@ -770,8 +770,17 @@ __device__ __forceinline__ void recover_rows_bulk(const uint8_t *__restrict__ co
         fence_async_smem();
         __syncthreads();
         if (tid == 0) {
-            const uint32_t bytes = (uint32_t)min((int64_t)kRecoverTileChunks, n - base) * 32u;
-            bulk_s2g(ob + base * 32, buf, bytes);
+            const int64_t cnt = min((int64_t)kRecoverTileChunks, n - base);
+            if (ld == cols) {
+                bulk_s2g(ob + base * 32, buf, (uint32_t)cnt * 32u);
+            } else { // rows with a leading dimension: one store per piece of a row inside the tile, one group per tile
+                for (int64_t c = base; c < base + cnt;) {
+                    const int64_t row = c / cpr, col = c - row * cpr;
+                    const int64_t seg = min(cpr - col, base + cnt - c);
+                    bulk_s2g(ob + (row * ld + col * 16) * 2, buf + (c - base) * 32, (uint32_t)seg * 32u);
+                    c += seg;
+                }
+            }
             bulk_commit();
         }
     }
