@@ -119,6 +119,24 @@ __device__ __forceinline__ float exp_ratio(float d)
     return r;
 }
 
+// exp(d) - 1 for the K3 term.  |d| <= 0.5 (an actor a few updates away from its reference): the Taylor series to
+// degree 9 by FMAs, relative error about 2e-7 without the cancellation of exp(d) - 1; beyond that exp_ratio(d) - 1,
+// whose relative error stays below 1e-6 there.  About half the instructions of expm1f.
+__device__ __forceinline__ float expm1_k3(float d)
+{
+    if (fabsf(d) > 0.5f)
+        return exp_ratio(d) - 1.0f;
+    float p = 2.7557319e-6f;       // 1/9!
+    p = fmaf(p, d, 2.4801587e-5f); // 1/8!
+    p = fmaf(p, d, 1.9841270e-4f); // 1/7!
+    p = fmaf(p, d, 1.3888889e-3f); // 1/6!
+    p = fmaf(p, d, 8.3333333e-3f); // 1/5!
+    p = fmaf(p, d, 4.1666667e-2f); // 1/4!
+    p = fmaf(p, d, 1.6666667e-1f); // 1/3!
+    p = fmaf(p, d, 0.5f);          // 1/2!
+    return fmaf(p * d, d, d);
+}
+
 // VAR selects the score variants of the component ablations: 0 = the coefficient omega itself; 1 = chi_t r_t
 // replaced by 1 in the policy contribution; 2 = the advantage-only signal m_t A.
 template <bool KL, bool EXTRA, int VAR>
@@ -187,7 +205,7 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
             } else {
                 v = (VAR == 1) ? (m ? coef : 0.0f) : ((m && c) ? coef * r[i] : 0.0f);
                 if (KL && m)
-                    v += kl * (-expm1f(rf[i] - s[i]));
+                    v += kl * (-expm1_k3(rf[i] - s[i]));
             }
             w[i] = v;
         }
@@ -352,7 +370,7 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_packed_kernel(const
             chi |= (uint32_t)c << (8 * i);
             float v = (m && c) ? coef * r[i] : 0.0f;
             if (KL && m)
-                v += kl * (-expm1f(rf[i] - s[i]));
+                v += kl * (-expm1_k3(rf[i] - s[i]));
             w[i] = v;
         }
         if (cnt[j] == 4) {
@@ -417,7 +435,7 @@ __device__ __forceinline__ float fused_omega(float s, float o, float rf, bool m,
     const bool c = (A >= 0.0f) ? (r <= hi) : (r >= lo);
     float v = (m && c) ? coef * r : 0.0f;
     if (kl != 0.0f && m)
-        v += kl * (-expm1f(rf - s));
+        v += kl * (-expm1_k3(rf - s));
     return v;
 }
 

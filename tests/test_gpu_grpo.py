@@ -226,3 +226,18 @@ def test_random_rollouts_and_microbatch_slices(seed):
         n_rows = int(rng.integers(1, ro.n_resp - off + 1))
         got = G.grpo_coeffs(ro, resp_offset=off, n_rows=n_rows, N_norm=ro.n_valid, clip_eps=clip, beta=beta)
         check_coeffs(ro, got, resp_offset=off, beta=beta, clip_eps=clip)
+
+
+def test_k3_term_alone_over_a_wide_range_of_log_ratios():
+    """Zero advantages (equal rewards): omega is the K3 term only, beta/N * (1 - exp(s_ref - s)); it must hold 1e-5
+    relative from |s_ref - s| = 1e-6 (no cancellation) to 30 (no overflow), on both sides of the 0.5 switch."""
+    ro = synth.rollout(43, 2, 4, 1024, rewards="uniform", equal_group_fraction=1.0)
+    mag = np.logspace(-6, np.log10(30.0), ro.logp_new.size // 2, dtype=np.float64)
+    d = np.concatenate([mag, -mag]).astype(np.float32).reshape(ro.logp_new.shape)
+    d.reshape(-1)[[0, 1, 2, 3]] = np.float32([0.5, -0.5, np.nextafter(np.float32(0.5), np.float32(1)), 0.0])
+    ro.logp_ref[:] = ro.logp_new + d
+    got = G.grpo_coeffs(ro, N_norm=ro.n_valid, beta=0.25)
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    assert np.all(adv == 0)
+    w, _, _ = oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, ro.logp_ref, ro.mask, N_norm=ro.n_valid, beta=0.25)
+    assert G.rel_err(got["omega"], w).max() <= RTOL
