@@ -29,6 +29,8 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     __shared__ uint32_t sm_tab[2][kScaleTableWords]; // scale tables: [0] Q = 448, [1] Q = 127
     if (FMT < 0 || FMT == HILORE_FMT_E4M3FN_BLK) fill_scale_table<HILORE_FMT_E4M3FN_BLK>(sm_tab[0]);
     if (FMT < 0 || FMT == HILORE_FMT_INT8_BLK) fill_scale_table<HILORE_FMT_INT8_BLK>(sm_tab[1]);
+    grid_dependency_wait();    // everything above touched shared memory only
+    grid_dependency_release(); // the next kernel's CTAs may take the place of ours as they finish
     __shared__ uint64_t sm_share[2]; // this CTA's multipliers for its share of a unit's rows
     if (threadIdx.x == 0) {
         sm_share[0] = ((uint64_t)blockIdx.x << 32) / gridDim.x;
@@ -59,6 +61,8 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_k
 {
     __shared__ __align__(128) uint8_t sm_out[kRecoverStageBytes];
     __shared__ UnitStage stage;
+    grid_dependency_wait();
+    grid_dependency_release();
     stage_units(wk, true, stage);
     __syncthreads();
     uint32_t tile = 0;
@@ -149,7 +153,20 @@ template <typename K> static int launch_one(K kernel, CodecWork wk, int64_t tota
     int64_t grid = (int64_t)sm_count() * ctas_per_sm(kernel, kCodecThreads, 0, 2);
     if (grid > total_rows)
         grid = total_rows;
-    kernel<<<(unsigned)grid, kCodecThreads, 0, st>>>(wk);
+    // Programmatic dependent launch: the CTAs of this kernel may become resident while the previous kernel of the
+    // stream drains; they wait (griddepcontrol.wait) before their first access to global memory.
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kCodecThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, wk) != cudaSuccess)
+        return HILORE_CUDA;
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
 }
 

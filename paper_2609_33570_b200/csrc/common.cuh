@@ -48,6 +48,12 @@ __device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
+// Programmatic dependent launch: block until the kernels this one depends on have completed and their writes are
+// visible (a no-op when the kernel was launched without the attribute); and tell the next kernel of the stream that
+// it may start to become resident.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- packed conversions ----
 // Two fp32 -> two E4M3FN codes, round to nearest even, saturating at +-448; `lo` lands in the low byte.
 __device__ __forceinline__ uint32_t cvt_e4m3x2(float hi, float lo)
