@@ -1,33 +1,59 @@
-"""Bandwidth sweep of the single-unit entry points (`python -m paper_2609_33570_b200.sweep`).
+"""Bandwidth sweep of the single-unit entry points and the auxiliary kernels (`python bench_sweep.py`).
 
 Units [rows, cols] bf16 of 1 MiB ... 4 GiB (row width 4096 by default), compress then recover, and the
 coefficient kernel over 2^16 ... 2^24 slots at G = 16.  Each point is timed with CUDA events over `reps`
 calls that rotate through a pool of distinct buffers larger than L2, so the numbers are HBM numbers.
-Prints one JSON line per point.
+Prints one JSON line per point.  `bench.py` imports the point functions for the per-config legs of its line.
+
+`--case codec|coeffs|exposure` runs one small single-kernel case a few times and exits: inputs larger than
+L2, well under a few GB on the device, a handful of launches -- the cases the profiler captures under
+`profiles/` were taken on.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import os
+import sys
 
 import torch
 
-from . import api, synth
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+from paper_2609_33570_b200 import api, synth  # noqa: E402
 
 L2_BYTES = 126 << 20
 
 
-def _time(fn_list, reps):
-    for f in fn_list[: min(len(fn_list), 3)]:
+def time_calls(fn_list, reps, warm=3):
+    """Rotate through `fn_list` for `reps` calls.  loop_ms: CUDA events around the whole back-to-back loop, per call
+    (the throughput figure).  device_us: median over calls of an event pair around each single call (what the GPU
+    spends on one call, launch gaps of the stream included).  host_us: wall clock the host spends issuing one call
+    (binding + launch), measured without synchronising -- a call is launch-bound when host_us exceeds device_us."""
+    import time
+    for f in fn_list[: min(len(fn_list), warm)]:
         f()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
+    t0 = time.perf_counter()
     for i in range(reps):
         fn_list[i % len(fn_list)]()
+    host = (time.perf_counter() - t0) / reps
     e1.record()
     torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / reps
+    loop_ms = e0.elapsed_time(e1) / reps
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for i in range(reps):
+        pairs[i][0].record()
+        fn_list[i % len(fn_list)]()
+        pairs[i][1].record()
+    torch.cuda.synchronize()
+    dev = sorted(a.elapsed_time(b) for a, b in pairs)[reps // 2]
+    return {"loop_ms": loop_ms, "device_us": dev * 1e3, "host_us": host * 1e6}
+
+
+def _time(fn_list, reps):
+    return time_calls(fn_list, reps)["loop_ms"]
 
 
 def codec_point(rows, cols, fmt, reps, with_rms=True, max_pool_bytes=6 << 30):
@@ -49,28 +75,51 @@ def codec_point(rows, cols, fmt, reps, with_rms=True, max_pool_bytes=6 << 30):
            for i in range(pool)]
     n = rows * cols
     nbytes = 3 * n + (4 * n // 64 if block else 0)
-    tc, tr = _time(comp, reps), _time(rec, reps)
+    dc, dr = time_calls(comp, reps), time_calls(rec, reps)
+    tc, tr = dc["loop_ms"], dr["loop_ms"]
     return {"kernel": "codec", "rows": rows, "cols": cols, "fmt": fmt, "unit_mib": unit_bytes / 2 ** 20, "pool": pool,
             "compress_us": tc * 1e3, "compress_gbs": (nbytes + (4 * rows if with_rms else 0)) / tc / 1e6,
-            "recover_us": tr * 1e3, "recover_gbs": nbytes / tr / 1e6}
+            "compress_device_us": dc["device_us"], "compress_host_us": dc["host_us"],
+            "recover_us": tr * 1e3, "recover_gbs": nbytes / tr / 1e6,
+            "recover_device_us": dr["device_us"], "recover_host_us": dr["host_us"]}
 
 
-def coeffs_point(log2_slots, reps, G=16, T=1024):
+def coeffs_point(log2_slots, reps, G=16, T=1024, beta=0.0):
+    """hilore_grpo_coeffs over 2^log2_slots slots (13 B/slot; 17 with the K3 term, beta != 0)."""
     n_resp = max(G, (1 << log2_slots) // T)
     slots = n_resp * T
-    pool = max(1, min(8, -(-3 * L2_BYTES // (slots * 13))))
+    bps = 17 if beta else 13
+    pool = max(1, min(8, -(-3 * L2_BYTES // (slots * bps))))
     gen = torch.Generator(device="cuda")
     gen.manual_seed(1)
     lp = [torch.randn((n_resp, T), generator=gen, device="cuda") * 0.5 - 1.5 for _ in range(pool)]
     lo = [x + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.05 for x in lp]
+    lr = [x + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.05 for x in lp] if beta else [None] * pool
     mask = torch.ones((n_resp, T), dtype=torch.uint8, device="cuda")
     rewards = (torch.rand(n_resp, generator=gen, device="cuda") < 0.5).float()
     omega = [torch.empty_like(x) for x in lp]
-    fns = [lambda i=i: api.hilore_grpo_coeffs(rewards, n_resp, G, 0, n_resp, T, lp[i], lo[i], None, mask, slots, None, 0.2,
-                                              0.0, 1e-6, None, omega[i], None, None) for i in range(pool)]
-    t = _time(fns, reps)
-    return {"kernel": "grpo_coeffs", "slots": slots, "pool": pool, "us": t * 1e3, "tokens_per_s": slots / t * 1e3,
-            "gbs": 13 * slots / t / 1e6}
+    fns = [lambda i=i: api.hilore_grpo_coeffs(rewards, n_resp, G, 0, n_resp, T, lp[i], lo[i], lr[i], mask, slots, None, 0.2,
+                                              beta, 1e-6, None, omega[i], None, None) for i in range(pool)]
+    d = time_calls(fns, reps)
+    t = d["loop_ms"]
+    return {"kernel": "grpo_coeffs", "slots": slots, "beta": beta, "pool": pool, "us": t * 1e3, "device_us": d["device_us"],
+            "host_us": d["host_us"], "tokens_per_s": slots / t * 1e3, "gbs": bps * slots / t / 1e6}
+
+
+def coeffs_rollout_point(ro, reps):
+    """hilore_grpo_coeffs over a whole host-drawn rollout batch (masks and rewards as drawn), N on the device."""
+    dev = lambda a: torch.from_numpy(a).cuda()
+    R, ln, lo, mk = dev(ro.rewards), dev(ro.logp_new), dev(ro.logp_old), dev(ro.mask)
+    omega = [torch.empty_like(ln) for _ in range(3)]
+    n = torch.zeros(1, dtype=torch.int64, device="cuda")
+    api.hilore_mask_count(mk, mk.numel(), n)
+    fns = [lambda i=i: api.hilore_grpo_coeffs(R, ro.n_resp, ro.G, 0, ro.n_resp, ro.T, ln, lo, None, mk, 0, n, 0.2, 0.0, 1e-6,
+                                              None, omega[i], None, None) for i in range(3)]
+    d = time_calls(fns, reps)
+    slots = ro.n_resp * ro.T
+    t = d["loop_ms"]
+    return {"kernel": "grpo_coeffs", "slots": slots, "valid": ro.n_valid, "us": t * 1e3, "device_us": d["device_us"],
+            "tokens_per_s": slots / t * 1e3, "valid_tokens_per_s": ro.n_valid / t * 1e3, "gbs": 13 * slots / t / 1e6}
 
 
 def relerr_point(rows, cols, fmt, reps):
@@ -91,13 +140,14 @@ def relerr_point(rows, cols, fmt, reps):
             "gbs": 2 * rows * cols / t / 1e6, "e": e.item()}
 
 
-def exposure_point(log2_tok, U, reps):
-    """hilore_unit_exposure over n_tok tokens and U units: n_tok * (5 + 4 U) bytes."""
+def exposure_point(log2_tok, U, reps, masked_fraction=0.8):
+    """hilore_unit_exposure over n_tok tokens (a share `masked_fraction` of them valid) and U units:
+    n_tok * (5 + 4 U) bytes."""
     n_tok = 1 << log2_tok
     gen = torch.Generator(device="cuda")
     gen.manual_seed(5)
     omega = torch.randn(n_tok, generator=gen, device="cuda") * 1e-5
-    mask = (torch.rand(n_tok, generator=gen, device="cuda") < 0.8).to(torch.uint8)
+    mask = (torch.rand(n_tok, generator=gen, device="cuda") < masked_fraction).to(torch.uint8)
     pool = max(1, min(4, -(-3 * L2_BYTES // (n_tok * 4 * U))))
     rms = [torch.rand((U, n_tok), generator=gen, device="cuda") + 0.5 for _ in range(pool)]
     out = torch.zeros(U, device="cuda")
@@ -105,9 +155,10 @@ def exposure_point(log2_tok, U, reps):
     ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
     fns = [lambda i=i: api.hilore_unit_exposure(omega, mask, 1, n_tok, rms[i], U, n_tok, 0, 1e-8, out, None, ws, nws)
            for i in range(pool)]
-    t = _time(fns, reps)
-    return {"kernel": "unit_exposure", "n_tok": n_tok, "U": U, "pool": pool, "us": t * 1e3,
-            "gbs": n_tok * (5 + 4 * U) / t / 1e6}
+    d = time_calls(fns, reps)
+    t = d["loop_ms"]
+    return {"kernel": "unit_exposure", "n_tok": n_tok, "U": U, "pool": pool, "us": t * 1e3, "device_us": d["device_us"],
+            "host_us": d["host_us"], "gbs": n_tok * (5 + 4 * U) / t / 1e6}
 
 
 def coeffs_packed_point(log2_tokens, reps, G=8, mean_len=2048):
@@ -224,6 +275,55 @@ def plan_points(model="7B", rows=16384, layers=28, reps=5):
                     "gbs": nbytes / t / 1e6})
     return out
 
+# ---------------------------------------------------------------- small single-kernel cases (profiler captures)
+def codec_case(rows, cols, fmt, reps, units, rms=True, codes_on=True, recover=True):
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(0)
+    block = 0 if fmt == api.FMT_E4M3FN_RAW else 64
+    xs = [synth.activation_unit_device(gen, rows, cols) for _ in range(units)]
+    codes = [torch.empty((rows, cols), dtype=torch.uint8, device="cuda") for _ in range(units)]
+    scales = [torch.empty((rows, max(cols // 64, 1)), dtype=torch.float32, device="cuda") for _ in range(units)]
+    outs = [torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda") for _ in range(units)]
+    rms_buf = torch.empty((units, rows), dtype=torch.float32, device="cuda")
+    for _ in range(reps):
+        for i in range(units):
+            api.hilore_compress(xs[i], rows, cols, cols, fmt, block, codes[i] if codes_on else None,
+                                scales[i] if (block and codes_on) else None, rms_buf[i] if (rms or not codes_on) else None)
+        for i in range(units if recover else 0):
+            api.hilore_recover(codes[i], scales[i] if block else None, rows, cols, fmt, block, outs[i], cols)
+    torch.cuda.synchronize()
+
+
+def coeffs_case(log2_slots, reps, beta=0.0, G=16, T=1024):
+    n_resp = (1 << log2_slots) // T
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1)
+    lp = torch.randn((n_resp, T), generator=gen, device="cuda") * 0.5 - 1.5
+    lo = lp + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.05
+    lr = lp + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.05 if beta else None
+    mask = torch.ones((n_resp, T), dtype=torch.uint8, device="cuda")
+    rewards = (torch.rand(n_resp, generator=gen, device="cuda") < 0.5).float()
+    omega = torch.empty_like(lp)
+    for _ in range(reps):
+        api.hilore_grpo_coeffs(rewards, n_resp, G, 0, n_resp, T, lp, lo, lr, mask, n_resp * T, None, 0.2,
+                               beta, 1e-6, None, omega, None, None)
+    torch.cuda.synchronize()
+
+
+def exposure_case(log2_tok, U, reps):
+    n_tok = 1 << log2_tok
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    omega = torch.randn(n_tok, generator=gen, device="cuda") * 1e-5
+    mask = (torch.rand(n_tok, generator=gen, device="cuda") < 0.8).to(torch.uint8)
+    rms = torch.rand((U, n_tok), generator=gen, device="cuda") + 0.5
+    out = torch.zeros(U, device="cuda")
+    nws = api.hilore_workspace_bytes(U, n_tok)
+    ws = torch.empty(nws, dtype=torch.uint8, device="cuda")
+    for _ in range(reps):
+        api.hilore_unit_exposure(omega, mask, 1, n_tok, rms, U, n_tok, 0, 1e-8, out, None, ws, nws)
+    torch.cuda.synchronize()
+
 
 def main():
     ap = argparse.ArgumentParser()
@@ -236,7 +336,25 @@ def main():
     ap.add_argument("--no-coeffs", action="store_true")
     ap.add_argument("--no-rms", action="store_true", help="compress without the fused token RMS")
     ap.add_argument("--plan-table", action="store_true", help="only the 7B-shaped table under several candidate plans")
+    ap.add_argument("--case", choices=["codec", "coeffs", "exposure"], help="run one small single-kernel case and exit")
+    ap.add_argument("--rows", type=int, default=8192)
+    ap.add_argument("--fmt", type=int, default=api.FMT_E4M3FN_BLK)
+    ap.add_argument("--units", type=int, default=2)
+    ap.add_argument("--log2-slots", type=int, default=24)
+    ap.add_argument("--beta", type=float, default=0.0)
+    ap.add_argument("--U", type=int, default=12)
+    ap.add_argument("--stats-only", action="store_true", help="--case codec: token RMS only, no codes")
+    ap.add_argument("--no-recover", action="store_true")
     a = ap.parse_args()
+    if a.case == "codec":
+        codec_case(a.rows, a.cols, a.fmt, a.reps, a.units, rms=not a.no_rms, codes_on=not a.stats_only, recover=not a.no_recover)
+    elif a.case == "coeffs":
+        coeffs_case(a.log2_slots, a.reps, a.beta)
+    elif a.case == "exposure":
+        exposure_case(a.log2_slots, a.U, a.reps)
+    if a.case:
+        print("done")
+        return
     if a.plan_table:
         for p in plan_points():
             print(json.dumps(p), flush=True)
@@ -254,7 +372,8 @@ def main():
             torch.cuda.empty_cache()
     if not a.no_coeffs:
         for ls in range(16, 25):
-            print(json.dumps(coeffs_point(ls, a.reps)), flush=True)
+            for beta in (0.0, 1e-3):
+                print(json.dumps(coeffs_point(ls, a.reps, beta=beta)), flush=True)
         for fmt in a.fmts:
             print(json.dumps(relerr_point(65536, 8960, fmt, a.reps)), flush=True)
         for ls, U in ((13, 84), (17, 84), (20, 84), (24, 12)):

@@ -56,89 +56,110 @@ struct CoeffArgs {
 
 constexpr int kCoeffThreads = 128;
 constexpr int kCoeffVec = 2;                                  // float4 groups per thread
-constexpr int kCoeffTile = kCoeffThreads * kCoeffVec * 4;     // 1024 slots of one response per CTA
+constexpr int kCoeffTile = kCoeffThreads * kCoeffVec * 4;     // 1024 slots of one response per CTA (generic kernel)
 
 // Mean and population standard deviation of the G rewards of one prompt group, in fp64 (one warp; every lane
-// returns the same values).  `equal` is set when all G rewards are the same number.
+// returns the same values).  One pass over the rewards shifted by the group's first one, d_j = R_j - R_0 (exact
+// in fp64): mean = R_0 + S1 / G, variance = (S2 - S1^2 / G) / G with S1 = sum d_j, S2 = sum d_j^2.  Because
+// d_0 = 0 the subtraction loses at most a factor G of the 2^-53 relative precision; and all rewards are the same
+// number exactly when S2 == 0, which is the test for an equal-reward group.
 struct GroupStats {
-    double mu, sigma;
+    double r0, mu, sigma; // mu is the mean of the shifted rewards
     bool equal;
 };
 
 __device__ __forceinline__ GroupStats group_stats(const float *R, int G, int lane)
 {
-    float lo = INFINITY, hi = -INFINITY;
-    double sum = 0.0;
-    for (int j = lane; j < G; j += 32) {
-        const float v = __ldg(R + j);
-        lo = fminf(lo, v);
-        hi = fmaxf(hi, v);
-        sum += (double)v;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
-        hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
-    }
-    sum = warp_sum(sum);
     GroupStats g;
-    g.equal = lo == hi;
-    g.mu = sum / (double)G;
+    g.r0 = (double)__ldg(R);
+    double s1 = 0.0, s2 = 0.0;
+    for (int j = lane; j < G; j += 32) {
+        const double d = (double)__ldg(R + j) - g.r0;
+        s1 += d;
+        s2 = fma(d, d, s2);
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    g.equal = s2 == 0.0;
+    g.mu = 0.0;
     g.sigma = 0.0;
     if (g.equal)
         return g;
-    double var = 0.0;
-    for (int j = lane; j < G; j += 32) {
-        const double d = (double)__ldg(R + j) - g.mu;
-        var += d * d;
-    }
-    var = warp_sum(var) / (double)G;
-    g.sigma = sqrt(var);
+    g.mu = s1 / (double)G;
+    g.sigma = sqrt(fmax((s2 - s1 * g.mu) / (double)G, 0.0));
     return g;
 }
 
 // Advantage of a response with reward `r`: exactly zero in an equal-reward group, whatever the rounding of the mean.
 __device__ __forceinline__ float advantage_of(const GroupStats &g, float r, float adv_eps)
 {
-    return g.equal ? 0.0f : (float)(((double)r - g.mu) / (g.sigma + (double)adv_eps));
+    return g.equal ? 0.0f : (float)((((double)r - g.r0) - g.mu) / (g.sigma + (double)adv_eps));
 }
 
 // Advantage of response `resp`, from the G rewards of its prompt group (one warp).
-__device__ float group_advantage(const float *rewards, int64_t resp, int G, float adv_eps, int lane)
+__device__ __forceinline__ float group_advantage(const float *rewards, int64_t resp, int G, float adv_eps, int lane)
 {
     const GroupStats g = group_stats(rewards + (resp / G) * G, G, lane);
     return advantage_of(g, __ldg(rewards + resp), adv_eps);
 }
 
+constexpr float kLog2e = 1.4426950408889634f;
+
 // exp(d) for the importance ratio: one multiplication and one ex2.approx (relative error |d| * 2^-24 + 2^-22:
 // 3e-7 for the |d| < 1 of an actor update, below 6e-6 over the whole range where the result is a normal number).
-__device__ __forceinline__ float exp_ratio(float d)
+__device__ __forceinline__ float ex2_approx(float x)
 {
     float r;
-    asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(d * 1.4426950408889634f));
+    asm("ex2.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
+__device__ __forceinline__ float exp_ratio(float d) { return ex2_approx(__fmul_rn(d, kLog2e)); }
 
-// exp(d) - 1 for the K3 term.  |d| <= 0.5 (an actor a few updates away from its reference): the Taylor series to
-// degree 9 by FMAs, relative error about 2e-7 without the cancellation of exp(d) - 1; beyond that exp_ratio(d) - 1,
-// whose relative error stays below 1e-6 there.  About half the instructions of expm1f.
+// exp(d) - 1 for the K3 term.  |d| <= 0.25 (an actor a few updates away from its reference): the Taylor series to
+// degree 6 by FMAs (the first dropped term is d^6 / 5040 of the result: 5e-8), no cancellation; beyond that
+// exp_ratio(d) - 1, whose relative error 2^-22 e^d / |e^d - 1| stays below 9e-7 there.
+constexpr float kK3Switch = 0.25f;
 __device__ __forceinline__ float expm1_k3(float d)
 {
-    if (fabsf(d) > 0.5f)
+    if (fabsf(d) > kK3Switch)
         return exp_ratio(d) - 1.0f;
-    float p = 2.7557319e-6f;       // 1/9!
-    p = fmaf(p, d, 2.4801587e-5f); // 1/8!
-    p = fmaf(p, d, 1.9841270e-4f); // 1/7!
-    p = fmaf(p, d, 1.3888889e-3f); // 1/6!
-    p = fmaf(p, d, 8.3333333e-3f); // 1/5!
-    p = fmaf(p, d, 4.1666667e-2f); // 1/4!
-    p = fmaf(p, d, 1.6666667e-1f); // 1/3!
-    p = fmaf(p, d, 0.5f);          // 1/2!
-    return fmaf(p * d, d, d);
+    float p = 1.3888889e-3f;        // 1/6!
+    p = fmaf(p, d, 8.3333333e-3f);  // 1/5!
+    p = fmaf(p, d, 4.1666667e-2f);  // 1/4!
+    p = fmaf(p, d, 1.6666667e-1f);  // 1/3!
+    p = fmaf(p, d, 0.5f);           // 1/2!
+    return fmaf(__fmul_rn(p, d), d, d);
+}
+// The same polynomial for two values at once (each lane rounded like the scalar form, so the bits agree).
+__device__ __forceinline__ uint64_t expm1_k3_poly_x2(uint64_t d)
+{
+    uint64_t p = f32x2_pack(1.3888889e-3f, 1.3888889e-3f);
+    p = f32x2_fma(p, d, f32x2_pack(8.3333333e-3f, 8.3333333e-3f));
+    p = f32x2_fma(p, d, f32x2_pack(4.1666667e-2f, 4.1666667e-2f));
+    p = f32x2_fma(p, d, f32x2_pack(1.6666667e-1f, 1.6666667e-1f));
+    p = f32x2_fma(p, d, f32x2_pack(0.5f, 0.5f));
+    return f32x2_fma(f32x2_mul(p, d), d, d);
 }
 
+// One coefficient, the defining sequence of operations (every kernel of this file produces these bits):
+//   r = exp_ratio(s - o);  chi = A >= 0 ? r <= hi : r >= lo;  policy = chi ? coef * r : 0   (coef = -A / N)
+//   omega = m ? fma(-beta / N, expm1_k3(s_ref - s), policy) : 0                              (K3 term if beta != 0)
 // VAR selects the score variants of the component ablations: 0 = the coefficient omega itself; 1 = chi_t r_t
 // replaced by 1 in the policy contribution; 2 = the advantage-only signal m_t A.
+template <int VAR = 0>
+__device__ __forceinline__ float omega_scalar(float s, float o, float rf, bool m, bool kl_on, float A, float coef, float nkl,
+                                              float hi, float lo, float &r, bool &c)
+{
+    r = exp_ratio(s - o);
+    c = (A >= 0.0f) ? (r <= hi) : (r >= lo);
+    float v = VAR == 2 ? A : (VAR == 1 ? coef : (c ? __fmul_rn(coef, r) : 0.0f));
+    if (kl_on && VAR != 2)
+        v = fmaf(nkl, expm1_k3(rf - s), v);
+    return m ? v : 0.0f;
+}
+
+// Generic kernel: one CTA of 128 threads per 1024 slots of one response, 128-bit accesses (T % 4 == 0, 16-byte
+// alignment).  Takes the shapes the warp-tile kernel below does not.
 template <bool KL, bool EXTRA, int VAR>
 __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid_constant__ CoeffArgs a)
 {
@@ -149,6 +170,7 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
     const int64_t row = row32;
     const int tid = threadIdx.x, lane = tid & 31;
     const int64_t rowbase = row * a.T;
+    grid_dependency_wait();
 
     // issue the token loads first; the group statistics below overlap with them
     float4 sn[kCoeffVec], so[kCoeffVec], sr[kCoeffVec];
@@ -165,8 +187,9 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
             mk[j] = __ldcs(reinterpret_cast<const unsigned int *>(a.mask + k));
         }
     }
+    grid_dependency_release();
 
-    __shared__ float s_adv, s_coef, s_kl;
+    __shared__ float s_adv, s_coef, s_nkl;
     if (tid < 32) { // the per-response scalars, fp64 arithmetic once per CTA
         const float A = group_advantage(a.rewards, a.resp_offset + row, a.G, a.adv_eps, lane);
         if (lane == 0) {
@@ -174,15 +197,14 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
             const double invN = N > 0 ? 1.0 / (double)N : 0.0;
             s_adv = A;
             s_coef = (float)(-(double)A * invN); // omega = coef * r on the unclipped branch
-            s_kl = (float)((double)a.beta * invN);
+            s_nkl = -(float)((double)a.beta * invN);
             if (tt == 0 && a.adv_out)
                 a.adv_out[row] = A;
         }
     }
     __syncthreads();
-    const float A = s_adv, coef = s_coef, kl = s_kl;
+    const float A = s_adv, coef = s_coef, nkl = s_nkl;
     const float hi = 1.0f + a.clip_eps, lo = 1.0f - a.clip_eps;
-    const bool pos = A >= 0.0f;
 
 #pragma unroll
     for (int j = 0; j < kCoeffVec; ++j) {
@@ -196,24 +218,158 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const bool m = ((mk[j] >> (8 * i)) & 0xFFu) != 0;
-            r[i] = exp_ratio(s[i] - o[i]);
-            const bool c = pos ? (r[i] <= hi) : (r[i] >= lo);
+            bool c;
+            w[i] = omega_scalar<VAR>(s[i], o[i], KL ? rf[i] : 0.0f, m, KL, A, coef, nkl, hi, lo, r[i], c);
             chi |= (uint32_t)c << (8 * i);
-            float v;
-            if (VAR == 2) {
-                v = m ? A : 0.0f;
-            } else {
-                v = (VAR == 1) ? (m ? coef : 0.0f) : ((m && c) ? coef * r[i] : 0.0f);
-                if (KL && m)
-                    v += kl * (-expm1_k3(rf[i] - s[i]));
-            }
-            w[i] = v;
         }
         const int64_t k = rowbase + t0[j];
         __stcs(reinterpret_cast<float4 *>(a.omega + k), make_float4(w[0], w[1], w[2], w[3]));
         if (EXTRA) {
             if (a.ratio) __stcs(reinterpret_cast<float4 *>(a.ratio + k), make_float4(r[0], r[1], r[2], r[3]));
             if (a.clip_mask) __stcs(reinterpret_cast<unsigned int *>(a.clip_mask + k), chi);
+        }
+    }
+}
+
+// ---- the fast path: one WARP per tile of kWarpIters * 256 slots of one response, no CTA barrier
+// Tile and register budget, measured on B200 at 2^24 slots (13 B/slot; 17 with the K3 term): two pieces of 256
+// slots per warp and at most 80 registers (six CTAs per SM) give 34.0 / 44.3 us (6.4 TB/s both); one piece 39.7 /
+// 48.4, four pieces 34.3 / 48.1, the unconstrained 87-register build 36.1 / 47.4.
+#ifndef HILORE_COEFF_IT
+#define HILORE_COEFF_IT 2
+#endif
+#ifndef HILORE_COEFF_MINB
+#define HILORE_COEFF_MINB 6
+#endif
+#ifndef HILORE_COEFF_MINB_KL
+#define HILORE_COEFF_MINB_KL 6
+#endif
+constexpr int kWarpIters = HILORE_COEFF_IT;
+constexpr int kWarpTile = kWarpIters * 256;
+
+// Eight consecutive slots of one lane.  The subtractions, the scaling by log2(e), the product with -A / N and the
+// K3 polynomial run on packed fp32 pairs (one instruction per two slots, each lane rounded as the scalar
+// operation would be); ex2.approx, the clip compare and the selects are per slot.  Results are bit for bit those
+// of omega_scalar.  POS: the sign of the advantage (uniform over the warp), which fixes the side of the clip test.
+template <bool KL, bool EXTRA, int VAR, bool POS>
+__device__ __forceinline__ void coeffs8(const uint32_t (&sn)[8], const uint32_t (&so)[8], const uint32_t (&sr)[8], uint2 mk,
+                                        float A, float coef, float nkl, float hi, float lo, uint32_t (&w)[8],
+                                        uint32_t (&rr)[8], uint2 &chi)
+{
+    const uint64_t l2e = f32x2_pack(kLog2e, kLog2e), coef2 = f32x2_pack(coef, coef);
+    float v[8];
+    uint32_t cb[8];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const uint64_t s2 = u32x2_pack(sn[2 * e], sn[2 * e + 1]), o2 = u32x2_pack(so[2 * e], so[2 * e + 1]);
+        float x0, x1;
+        f32x2_unpack(f32x2_mul(f32x2_sub(s2, o2), l2e), x0, x1);
+        const float r0 = ex2_approx(x0), r1 = ex2_approx(x1);
+        const bool c0 = POS ? (r0 <= hi) : (r0 >= lo), c1 = POS ? (r1 <= hi) : (r1 >= lo);
+        if (VAR == 0) {
+            float p0, p1;
+            f32x2_unpack(f32x2_mul(coef2, f32x2_pack(r0, r1)), p0, p1);
+            v[2 * e] = c0 ? p0 : 0.0f;
+            v[2 * e + 1] = c1 ? p1 : 0.0f;
+        } else {
+            v[2 * e] = v[2 * e + 1] = VAR == 2 ? A : coef;
+        }
+        if (EXTRA) {
+            rr[2 * e] = __float_as_uint(r0);
+            rr[2 * e + 1] = __float_as_uint(r1);
+            cb[2 * e] = c0;
+            cb[2 * e + 1] = c1;
+        }
+    }
+    if (KL && VAR != 2) {
+        const uint64_t nkl2 = f32x2_pack(nkl, nkl);
+        float big = 0.0f; // largest |s_ref - s| of the eight
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const uint64_t d2 = f32x2_sub(u32x2_pack(sr[2 * e], sr[2 * e + 1]), u32x2_pack(sn[2 * e], sn[2 * e + 1]));
+            float d0, d1;
+            f32x2_unpack(d2, d0, d1);
+            big = fmaxf(big, fmaxf(fabsf(d0), fabsf(d1)));
+            f32x2_unpack(f32x2_fma(nkl2, expm1_k3_poly_x2(d2), f32x2_pack(v[2 * e], v[2 * e + 1])), v[2 * e], v[2 * e + 1]);
+        }
+        if (!(big <= kK3Switch)) { // rare (also taken for NaN): some slot is beyond the polynomial's range
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                float r;
+                bool c;
+                v[e] = omega_scalar<VAR>(__uint_as_float(sn[e]), __uint_as_float(so[e]), __uint_as_float(sr[e]), true, true, A,
+                                         coef, nkl, hi, lo, r, c);
+            }
+        }
+    }
+    if (mk.x != 0x01010101u || mk.y != 0x01010101u) { // some slot of the eight is masked out
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t byte = ((e < 4 ? mk.x : mk.y) >> (8 * (e & 3))) & 0xFFu;
+            v[e] = byte != 0 ? v[e] : 0.0f;
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) w[e] = __float_as_uint(v[e]);
+    if (EXTRA) {
+        chi.x = cb[0] | (cb[1] << 8) | (cb[2] << 16) | (cb[3] << 24);
+        chi.y = cb[4] | (cb[5] << 8) | (cb[6] << 16) | (cb[7] << 24);
+    }
+}
+
+// Each warp owns one tile: its loads (256-bit per lane and tensor) are issued first, the group statistics of its
+// response follow while they are in flight, then the arithmetic and the 256-bit stores.  Warps never wait for one
+// another.  Needs T % 8 == 0 and 32-byte aligned tensors (8-byte for the masks); launched with the
+// programmatic-serialization attribute, so a following launch of this library becomes resident while this one drains.
+template <bool KL, bool EXTRA, int VAR>
+__global__ void __launch_bounds__(kCoeffThreads, KL ? HILORE_COEFF_MINB_KL : HILORE_COEFF_MINB)
+    grpo_coeffs_warp_kernel(const __grid_constant__ CoeffArgs a, uint32_t total_tiles)
+{
+    const int lane = threadIdx.x & 31;
+    const uint32_t wt = blockIdx.x * (kCoeffThreads / 32) + (threadIdx.x >> 5);
+    if (wt >= total_tiles)
+        return;
+    const uint32_t tpr = (uint32_t)a.tiles_per_row;
+    const uint32_t row32 = tpr == 1 ? wt : wt / tpr;
+    const int tt = (int)(wt - row32 * tpr);
+    const int64_t row = row32, rowbase = row * a.T;
+    grid_dependency_wait();
+    uint32_t sn[kWarpIters][8], so[kWarpIters][8], sr[KL ? kWarpIters : 1][8];
+    uint2 mk[kWarpIters];
+    int64_t t0[kWarpIters];
+#pragma unroll
+    for (int i = 0; i < kWarpIters; ++i) {
+        t0[i] = (int64_t)tt * kWarpTile + i * 256 + lane * 8;
+        if (t0[i] < a.T) {
+            const int64_t k = rowbase + t0[i];
+            ld_global_256(a.logp_new + k, sn[i]);
+            ld_global_256(a.logp_old + k, so[i]);
+            if (KL) ld_global_256(a.logp_ref + k, sr[i]);
+            mk[i] = ld_global_64_stream(a.mask + k);
+        }
+    }
+    grid_dependency_release();
+    const float A = group_advantage(a.rewards, a.resp_offset + row, a.G, a.adv_eps, lane);
+    const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
+    const double invN = N > 0 ? 1.0 / (double)N : 0.0;
+    const float coef = (float)(-(double)A * invN);
+    const float nkl = -(float)((double)a.beta * invN);
+    if (tt == 0 && lane == 0 && a.adv_out)
+        a.adv_out[row] = A;
+    const float hi = 1.0f + a.clip_eps, lo = 1.0f - a.clip_eps;
+#pragma unroll
+    for (int i = 0; i < kWarpIters; ++i) {
+        if (t0[i] >= a.T)
+            continue;
+        uint32_t w[8], rr[8];
+        uint2 chi;
+        if (A >= 0.0f) coeffs8<KL, EXTRA, VAR, true>(sn[i], so[i], sr[KL ? i : 0], mk[i], A, coef, nkl, hi, lo, w, rr, chi);
+        else coeffs8<KL, EXTRA, VAR, false>(sn[i], so[i], sr[KL ? i : 0], mk[i], A, coef, nkl, hi, lo, w, rr, chi);
+        const int64_t k = rowbase + t0[i];
+        st_global_256(a.omega + k, w);
+        if (EXTRA) {
+            if (a.ratio) st_global_256(a.ratio + k, rr);
+            if (a.clip_mask) *reinterpret_cast<uint2 *>(a.clip_mask + k) = chi;
         }
     }
 }
@@ -333,7 +489,7 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_packed_kernel(const
     __syncthreads();
     const int seq_first = s_range[0], seq_end = s_range[1] + 1;
     const double invN = s_invN;
-    const float kl = (float)((double)a.beta * invN);
+    const float nkl = -(float)((double)a.beta * invN);
     const float hi = 1.0f + a.clip_eps, lo = 1.0f - a.clip_eps;
 
 #pragma unroll
@@ -365,13 +521,9 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_packed_kernel(const
                 coef = (float)(-(double)A * invN);
             }
             const bool m = ((mk[j] >> (8 * i)) & 0xFFu) != 0;
-            r[i] = exp_ratio(s[i] - o[i]);
-            const bool c = (A >= 0.0f) ? (r[i] <= hi) : (r[i] >= lo);
+            bool c;
+            w[i] = omega_scalar<0>(s[i], o[i], KL ? rf[i] : 0.0f, m, KL, A, coef, nkl, hi, lo, r[i], c);
             chi |= (uint32_t)c << (8 * i);
-            float v = (m && c) ? coef * r[i] : 0.0f;
-            if (KL && m)
-                v += kl * (-expm1_k3(rf[i] - s[i]));
-            w[i] = v;
         }
         if (cnt[j] == 4) {
             __stcs(reinterpret_cast<float4 *>(a.omega + k0[j]), make_float4(w[0], w[1], w[2], w[3]));
@@ -431,12 +583,9 @@ struct ExpArgs {
 // One coefficient, exactly as grpo_coeffs_kernel computes it (same expressions, same rounding).
 __device__ __forceinline__ float fused_omega(float s, float o, float rf, bool m, float A, float coef, float kl, float hi, float lo)
 {
-    const float r = exp_ratio(s - o);
-    const bool c = (A >= 0.0f) ? (r <= hi) : (r >= lo);
-    float v = (m && c) ? coef * r : 0.0f;
-    if (kl != 0.0f && m)
-        v += kl * (-expm1_k3(rf - s));
-    return v;
+    float r;
+    bool c;
+    return omega_scalar<0>(s, o, rf, m, kl != 0.0f, A, coef, -kl, hi, lo, r, c);
 }
 
 // FUSED: omega is not read but computed here from the log-probabilities (and written once, by the CTAs of the
@@ -683,13 +832,44 @@ static int launch_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, 
     a.omega = omega;
     a.ratio = ratio;
     a.clip_mask = clip_mask;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool kl = beta != 0.0f, extra = (ratio != nullptr) || (clip_mask != nullptr);
+    // programmatic dependent launch: the kernels wait (griddepcontrol.wait) before their first global access
+    cudaLaunchConfig_t cfg{};
+    cfg.blockDim = dim3(kCoeffThreads);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const bool wide = T % 8 == 0 && aligned(logp_new, 32) && aligned(logp_old, 32) && aligned(a.logp_ref, 32) &&
+                      aligned(omega, 32) && aligned(ratio, 32) && aligned(mask, 8) && aligned(clip_mask, 8);
+    if (wide) { // one warp per tile of kWarpTile slots
+        const int64_t tpr = (T + kWarpTile - 1) / kWarpTile;
+        const int64_t tiles = tpr * n_rows;
+        if (tpr > 0x7FFFFFFF || tiles > 0x7FFFFFFF)
+            return HILORE_SHAPE;
+        a.tiles_per_row = (int)tpr;
+        void (*kernel)(CoeffArgs, uint32_t) = nullptr;
+#define HILORE_PICK(V)                                                                                                  \
+    kernel = kl ? (extra ? grpo_coeffs_warp_kernel<true, true, V> : grpo_coeffs_warp_kernel<true, false, V>)            \
+                : (extra ? grpo_coeffs_warp_kernel<false, true, V> : grpo_coeffs_warp_kernel<false, false, V>)
+        if (variant == 0) { HILORE_PICK(0); }
+        else if (variant == 1) { HILORE_PICK(1); }
+        else { HILORE_PICK(2); }
+#undef HILORE_PICK
+        constexpr int kWarps = kCoeffThreads / 32;
+        cfg.gridDim = dim3((unsigned)((tiles + kWarps - 1) / kWarps));
+        if (cudaLaunchKernelEx(&cfg, kernel, a, (uint32_t)tiles) != cudaSuccess)
+            return HILORE_CUDA;
+        return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+    }
     const int64_t tpr = (T + kCoeffTile - 1) / kCoeffTile;
     const int64_t tiles = tpr * n_rows;
     if (tpr > 0x7FFFFFFF || tiles > 0x7FFFFFFF)
         return HILORE_SHAPE;
     a.tiles_per_row = (int)tpr;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool kl = beta != 0.0f, extra = (ratio != nullptr) || (clip_mask != nullptr);
     void (*kernel)(CoeffArgs) = nullptr;
 #define HILORE_PICK(V)                                                                                                  \
     kernel = kl ? (extra ? grpo_coeffs_kernel<true, true, V> : grpo_coeffs_kernel<true, false, V>)                      \
@@ -698,7 +878,9 @@ static int launch_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, 
     else if (variant == 1) { HILORE_PICK(1); }
     else { HILORE_PICK(2); }
 #undef HILORE_PICK
-    kernel<<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);
+    cfg.gridDim = dim3((unsigned)tiles);
+    if (cudaLaunchKernelEx(&cfg, kernel, a) != cudaSuccess)
+        return HILORE_CUDA;
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
 }
 

@@ -43,7 +43,8 @@ def sample_rows(rng, rows, n=24):
 def test_bench_step_1p5B_shaped_microbatch():
     """configs[1]: the exact object bench.py times (84 units, one launch per phase, all L)."""
     dev = torch.device("cuda", 0)
-    wl = bench.Workload(api, synth, seed=0, device=dev)
+    cfg = bench.CONFIGS[2]
+    wl = bench.Workload(api, synth, cfg, seed=0, device=dev)
     for t in wl.codes + wl.out:
         t.fill_(0xA5 if t.dtype == torch.uint8 else -1.0)
     wl.step(3)
@@ -57,7 +58,7 @@ def test_bench_step_1p5B_shaped_microbatch():
     # coefficients of microbatch 3, then exposure, psi and action of a sample of units, every expected value from the
     # oracle's own chain (its omega, its token RMS of the whole unit): a unit's exposure depends on that unit only
     ro = wl.ro
-    sl = slice(3 * bench.MB_RESP, 4 * bench.MB_RESP)
+    sl = slice(3 * cfg["mb_resp"], 4 * cfg["mb_resp"])
     adv = oracle.group_advantages(ro.rewards, ro.G)
     w, _, _ = oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=ro.n_valid)
     assert G.rel_err(wl.omega.cpu().numpy(), w).max() <= 1e-5
