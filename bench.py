@@ -589,7 +589,7 @@ def main():
     # sustained: the same step for at least `sustain_s` seconds, with its own clock record
     sustained = None
     if args.sustain_s > 0:
-        n_sus = max(args.steps, int(math.ceil(args.sustain_s * 1e3 / ms_step)))
+        n_sus = max(args.steps, int(math.ceil(1.1 * args.sustain_s * 1e3 / ms_step)))
         if rank == 0:
             sampler.start()
         ms_sus, _ = time_steps(wl, 0, n_sus, barrier, with_events=False)
