@@ -8,17 +8,24 @@
 namespace hilore {
 
 // Compress / token-RMS pass over rows [r0, r1) of one unit, specialised on what the unit asks for.
+// Iterations of bulk L2 prefetch run-ahead of the compress pass (16 KB of bf16 per iteration and CTA), by what
+// the pass writes.  Measured on B200 (TB/s at run-ahead 0 / 1 / 2 / 3): token RMS only, 7B-shaped table
+// 6.6 / 6.8 / 7.1 / 7.1; codes + scales + RMS, 7B-shaped table 6.2 / 6.6 / 6.4 / 6.0, 4 GiB unit 6.3 / 6.7 / 6.0;
+// the unscaled format on a 4 GiB unit 6.7 / 6.5 / 6.0; codes + scales only (post-forward encode) 6.7 / 6.4 / 6.1 /
+// 5.9: the more a pass writes, the sooner lines pulled in ahead of time are in the way of the written ones.
+constexpr int kPrefetchStats = 2, kPrefetchCodesRms = 1, kPrefetchCodesOnly = 0;
+
 template <int FMT>
-__device__ __forceinline__ void compress_unit(const hilore_unit &u, int op, int64_t r0, int64_t r1, float *sm, int pf,
+__device__ __forceinline__ void compress_unit(const hilore_unit &u, int op, int64_t r0, int64_t r1, int rpb, float *sm,
                                               const uint32_t *tab)
 {
     const uint16_t *x = static_cast<const uint16_t *>(u.x);
     if (op == OP_STATS)
-        compress_rows<HILORE_FMT_E4M3FN_RAW, false, true>(x, nullptr, nullptr, u.row_rms, u.cols, u.ld, r0, r1, sm, pf, tab);
+        compress_rows<HILORE_FMT_E4M3FN_RAW, false, true>(x, nullptr, nullptr, u.row_rms, u.cols, u.ld, r0, r1, rpb, sm, kPrefetchStats, tab);
     else if (u.row_rms != nullptr)
-        compress_rows<FMT, true, true>(x, u.codes, u.scales, u.row_rms, u.cols, u.ld, r0, r1, sm, pf, tab);
+        compress_rows<FMT, true, true>(x, u.codes, u.scales, u.row_rms, u.cols, u.ld, r0, r1, rpb, sm, FMT == HILORE_FMT_E4M3FN_RAW ? kPrefetchCodesOnly : kPrefetchCodesRms, tab);
     else
-        compress_rows<FMT, true, false>(x, u.codes, u.scales, nullptr, u.cols, u.ld, r0, r1, sm, pf, tab);
+        compress_rows<FMT, true, false>(x, u.codes, u.scales, nullptr, u.cols, u.ld, r0, r1, rpb, sm, kPrefetchCodesOnly, tab);
 }
 
 // FMT >= 0: every unit of the launch has this format (the common case; the hot loop is compiled for it).
@@ -31,19 +38,14 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     if (FMT < 0 || FMT == HILORE_FMT_INT8_BLK) fill_scale_table<HILORE_FMT_INT8_BLK>(sm_tab[1]);
     grid_dependency_wait();    // everything above touched shared memory only
     grid_dependency_release(); // the next kernel's CTAs may take the place of ours as they finish
-    __shared__ uint64_t sm_share[2]; // this CTA's multipliers for its share of a unit's rows
-    if (threadIdx.x == 0) {
-        sm_share[0] = ((uint64_t)blockIdx.x << 32) / gridDim.x;
-        sm_share[1] = ((uint64_t)(blockIdx.x + 1) << 32) / gridDim.x;
-    }
-    __syncthreads(); // scale tables and shares are filled
+    __syncthreads();           // scale tables are filled
     JobCursor cur;
-    DirectJob j;
-    while (next_job_direct(wk, cur, j, sm_share)) {
+    Job j;
+    while (next_job(wk, nullptr, false, cur, j, kBlockSumSlots)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
-        if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
-        else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[0]);
-        else compress_unit<HILORE_FMT_INT8_BLK>(j.u, j.op, j.r0, j.r1, sm_blocksum, wk.prefetch, sm_tab[1]);
+        if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[0]);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[0]);
+        else compress_unit<HILORE_FMT_INT8_BLK>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[1]);
     }
 }
 
@@ -68,11 +70,11 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_k
     uint32_t tile = 0;
     JobCursor cur;
     Job j;
-    while (next_job(wk, stage, cur, j)) {
-        const int fmt = FMT >= 0 ? FMT : j.u->fmt;
-        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(*j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
-        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(*j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
-        else recover_unit<HILORE_FMT_INT8_BLK>(*j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+    while (next_job(wk, &stage, true, cur, j, 0)) {
+        const int fmt = FMT >= 0 ? FMT : j.u.fmt;
+        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        else recover_unit<HILORE_FMT_INT8_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
     }
     if (threadIdx.x == 0)
         bulk_wait_all(); // every bulk store of this CTA is complete before it gives up its shared memory
@@ -137,10 +139,9 @@ static int check_unit(const hilore_unit &u, bool strict, bool need_x, bool need_
     return HILORE_OK;
 }
 
-// Iterations of bulk L2 prefetch run-ahead (16 KB of bf16 / 8 KB of codes per iteration and CTA).  Two is
-// the measured optimum on B200 for both passes; farther ahead the prefetched lines start to crowd the
-// written lines out of L2.
-constexpr int kPrefetchCompress = 2, kPrefetchRecover = 2;
+// Tiles of bulk L2 prefetch run-ahead of the recover pass (8 KB of codes per tile and CTA): one to three measure
+// alike on B200, none is 6 % slower.
+constexpr int kPrefetchRecover = 2;
 // Window of a unit that all CTAs sweep together (see next_job).  Measured on B200: a 4 GiB unit runs at
 // 5.5 / 6.2 TB/s (compress / recover) uncut, 6.0 / 6.3 TB/s in windows of 64-96 MB; below about 48 MB the
 // pieces per CTA become too short.
@@ -153,6 +154,17 @@ template <typename K> static int launch_one(K kernel, CodecWork wk, int64_t tota
     int64_t grid = (int64_t)sm_count() * ctas_per_sm(kernel, kCodecThreads, 0, 2);
     if (grid > total_rows)
         grid = total_rows;
+    wk.share_m = (1ull << 32) / (uint64_t)grid;
+    wk.share_rem = (uint32_t)((1ull << 32) % (uint64_t)grid);
+    // Rotation of the CTA index per window (see next_job): about 0.38 of the grid, coprime to it, so that the
+    // rotated indices of consecutive windows fall evenly.
+    wk.rot_step = 0;
+    if (grid > 2) {
+        uint32_t step = (uint32_t)(grid * 0.381966) | 1u;
+        auto gcd = [](uint32_t a, uint32_t b) { while (b) { const uint32_t t = a % b; a = b; b = t; } return a; };
+        while (gcd(step, (uint32_t)grid) != 1) step += 2;
+        wk.rot_step = step % (uint32_t)grid;
+    }
     // Programmatic dependent launch: the CTAs of this kernel may become resident while the previous kernel of the
     // stream drains; they wait (griddepcontrol.wait) before their first access to global memory.
     cudaLaunchConfig_t cfg{};
@@ -184,7 +196,7 @@ static int launch_codec(const CodecWork &wk, int64_t total_rows, int fmt, bool r
         default: return launch_one(recover_kernel<-1>, wk, total_rows, pf, st);
         }
     }
-    const int pf = kPrefetchCompress;
+    const int pf = 0; // the compress pass picks its run-ahead per unit (what it writes decides)
     switch (fmt) {
     case HILORE_FMT_E4M3FN_RAW: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, pf, st);
     case HILORE_FMT_E4M3FN_BLK: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, pf, st);

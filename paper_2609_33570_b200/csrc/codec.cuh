@@ -28,6 +28,9 @@ struct CodecWork {
     const uint8_t *action;    // a_u
     int prefetch;             // iterations of L2 prefetch run-ahead (0 = none)
     int64_t seg_bytes;        // size of the window all CTAs sweep together
+    uint64_t share_m;         // 2^32 = share_m * grid + share_rem
+    uint32_t share_rem;
+    uint32_t rot_step;        // rotation of the CTA index per window (0 for a single unit)
 };
 
 __device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
@@ -50,33 +53,30 @@ __device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
 
 
 // ---- work split ----
-// A unit is swept in equal segments of about `seg_bytes` of bf16 (units up to 1.5 x that size in one piece);
-// every CTA takes the same share of every segment: rows [n*c/nC, n*(c+1)/nC) of its n rows.  All CTAs
-// therefore work inside one window of memory at a time and finish together -- measured faster on B200 than
-// giving each CTA one large private slice of a unit or of the whole launch.
-//
-// With a microbatch of 84 units a CTA meets a new unit every few iterations, so what it costs to get to the
-// next unit counts: the descriptors and the gating decisions of a launch (at most kStageUnits units; the host
-// cuts longer tables into several launches) are staged in shared memory once, and a CTA's share of n rows is
-// (n * K) >> 32 with K = floor(c * 2^32 / nC) computed once per kernel -- the same partition for all CTAs
-// (consecutive CTAs share their boundary, the last one ends at n) for one multiplication instead of two 64-bit
-// divisions per unit.
+// What the CTAs of a launch share is a list of ITEMS per unit; CTA c' takes items [n*c'/nC, n*(c'+1)/nC) of every
+// window of n items, so that all CTAs work inside one window of memory at a time (measured faster on B200 than
+// one large private slice per CTA).  An item is a 16 KB piece (512 chunks: one iteration of the hot loops) of a
+// contiguous unit when no per-row result is wanted (encode without token RMS, recover): every CTA then runs whole
+// iterations only; otherwise a row (ragged ends of a CTA's rows take the predicated path).
+// c' is the CTA index rotated by a fixed step per window.  Without the rotation the same CTAs take the same
+// relative share of every unit of a microbatch; with it the shares move from unit to unit (measured on the 7B-shaped
+// table of 84 units: token-RMS capture 5.8 -> 7.1 TB/s, recovery 5.9 -> 6.3 TB/s; the size of the step does not
+// matter).  Nothing synchronises the CTAs between units, so only the total per CTA counts for the balance.
+// A CTA's share of n items is (n * K(c')) >> 32 with K(c) = floor(c * 2^32 / nC) = c * M + floor(c * rem / nC)
+// (M, rem from the host): one multiplication and a 32-bit division instead of two 64-bit divisions per window.
 constexpr int kStageUnits = 96;
+constexpr int kIterChunks = 2 * kCodecThreads;       // chunks one iteration of a CTA covers (16 KB of bf16)
+constexpr int kFlatCols = kIterChunks * 16;          // a 16 KB piece seen as one row of 8192 elements
 
 struct UnitStage {
     hilore_unit u[kStageUnits];
     int op[kStageUnits];
-    uint64_t k0, k1; // floor(c * 2^32 / nC), floor((c + 1) * 2^32 / nC) for this CTA c
 };
 
 // Stage the launch's units: what to do with each (OP_NONE if the launch is not gated into it or it lacks a
 // buffer the operation needs) and its descriptor.  `recover`: which of the two kernels is asking.
 __device__ __forceinline__ void stage_units(const CodecWork &wk, bool recover, UnitStage &st)
 {
-    if (threadIdx.x == 0) {
-        st.k0 = ((uint64_t)blockIdx.x << 32) / gridDim.x;
-        st.k1 = ((uint64_t)(blockIdx.x + 1) << 32) / gridDim.x;
-    }
     for (int t = threadIdx.x; t < wk.U; t += blockDim.x) {
         int op = unit_op(wk, t);
         if (recover ? (op != OP_RECOVER) : (op != OP_COMPRESS && op != OP_STATS))
@@ -95,91 +95,133 @@ __device__ __forceinline__ void stage_units(const CodecWork &wk, bool recover, U
     }
 }
 
-struct Job {
-    const hilore_unit *u; // in the shared-memory stage
-    int op;
-    int64_t r0, r1; // this CTA's rows of the current segment
-};
-
-struct JobCursor {
-    int ui = 0;          // next unit
-    int64_t seg_row = 0; // first row of the next segment of unit ui
-};
-
-__device__ __forceinline__ bool next_job(const CodecWork &wk, const UnitStage &st, JobCursor &cur, Job &j)
+__device__ __forceinline__ uint64_t share_multiplier(const CodecWork &wk, uint32_t c) // floor(c * 2^32 / nC), c <= nC
 {
-    for (; cur.ui < wk.U; ++cur.ui, cur.seg_row = 0) {
-        j.op = st.op[cur.ui];
-        if (j.op == OP_NONE)
-            continue;
-        j.u = &st.u[cur.ui];
-        const hilore_unit &u = *j.u;
-        // equal segments, as close to seg_bytes each as the unit's size allows
-        const int64_t unit_bytes = u.rows * u.cols * 2;
-        int64_t seg_rows = u.rows;
-        if (unit_bytes >= wk.seg_bytes + wk.seg_bytes / 2) {
-            const int64_t nseg = (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes;
-            seg_rows = (u.rows + nseg - 1) / nseg;
-        }
-        seg_rows = max((int64_t)gridDim.x, seg_rows);
-        while (cur.seg_row < u.rows) {
-            const int64_t s0 = cur.seg_row, n = min(seg_rows, u.rows - s0);
-            cur.seg_row += n;
-            if (n < (1ll << 31)) {
-                j.r0 = s0 + (int64_t)(((uint64_t)n * st.k0) >> 32);
-                j.r1 = s0 + (int64_t)(((uint64_t)n * st.k1) >> 32);
-            } else {
-                j.r0 = s0 + (n * (int64_t)blockIdx.x) / gridDim.x;
-                j.r1 = s0 + (n * (int64_t)(blockIdx.x + 1)) / gridDim.x;
-            }
-            if (j.r0 < j.r1)
-                return true; // the cursor already points at the next segment
-        }
-    }
-    return false;
+    return (uint64_t)c * wk.share_m + (c * wk.share_rem) / gridDim.x;
 }
 
-// The same walk without the stage: descriptors and gates are read from global memory at every unit.  The
-// compress kernel uses this form -- its 64-register budget is full, and the staged form costs it more in
-// register traffic inside the hot loop than it saves per unit.
-struct DirectJob {
+struct UnitPlan {
+    int64_t items;     // rows or 16 KB pieces
+    int64_t seg_items; // items per window
+    bool flat;         // items are 16 KB pieces
+    int tail_chunks;   // flat: chunks beyond the last whole piece
+};
+
+// `per_row`: a per-row result (token RMS) is wanted.
+__device__ __forceinline__ UnitPlan plan_unit(const CodecWork &wk, const hilore_unit &u, bool per_row)
+{
+    UnitPlan p;
+    int64_t item_bytes = u.cols * 2;
+    p.items = u.rows;
+    p.flat = false;
+    p.tail_chunks = 0;
+    if (u.ld == u.cols && !per_row) {
+        const int64_t chunks = u.rows * (u.cols >> 4);
+        p.items = chunks / kIterChunks;
+        p.tail_chunks = (int)(chunks - p.items * kIterChunks);
+        p.flat = true;
+        item_bytes = kFlatCols * 2;
+    }
+    // equal windows, as close to seg_bytes each as the unit's size allows (units up to 1.5 x that size in one piece)
+    const int64_t unit_bytes = p.items * item_bytes;
+    p.seg_items = p.items;
+    if (unit_bytes >= wk.seg_bytes + wk.seg_bytes / 2) {
+        const int64_t nseg = (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes;
+        p.seg_items = (p.items + nseg - 1) / nseg;
+    }
+    // a whole number of items per CTA and window, so that only a unit's last window is shared unevenly
+    const int64_t nC = gridDim.x;
+    p.seg_items = max((int64_t)1, (p.seg_items + nC / 2) / nC) * nC;
+    return p;
+}
+
+// One piece of work of a CTA: rows [r0, r1) of a unit (or of the 16 KB-piece view of it), in batches of
+// `rows_per_batch` rows where per-row sums are collected.
+struct Job {
     hilore_unit u;
     int op;
     int64_t r0, r1;
+    int rows_per_batch;
 };
 
-__device__ __forceinline__ bool next_job_direct(const CodecWork &wk, JobCursor &cur, DirectJob &j, const uint64_t *share)
+struct JobCursor {
+    int ui = 0;           // current unit
+    int64_t seg_item = 0; // first item of its next window
+    uint32_t rot = 0;     // rotation of the CTA index, advanced per window
+    bool tail_done = false;
+};
+
+// `st`: the staged descriptors (recover kernel), or nullptr: descriptors and gates are read from global memory at
+// every unit (compress kernel: its register budget is full, and the staged form cost more in the hot loop).
+__device__ __forceinline__ bool next_job(const CodecWork &wk, const UnitStage *st, bool recover, JobCursor &cur, Job &j, int slots)
 {
-    for (; cur.ui < wk.U; ++cur.ui, cur.seg_row = 0) {
-        j.op = unit_op(wk, cur.ui);
-        if (j.op != OP_COMPRESS && j.op != OP_STATS)
-            continue;
-        j.u = wk.units ? wk.units[cur.ui] : wk.single;
-        const hilore_unit &u = j.u;
-        const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
-        if ((j.op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (j.op == OP_STATS && (!u.x || !u.row_rms)))
-            continue; // the unit lacks a buffer this operation needs: leave it untouched
-        if (j.op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
-            j.u.row_rms = nullptr; // token magnitudes were collected at capture time
-        const int64_t unit_bytes = u.rows * u.cols * 2;
-        int64_t seg_rows = u.rows;
-        if (unit_bytes >= wk.seg_bytes + wk.seg_bytes / 2) {
-            const int64_t nseg = (unit_bytes + wk.seg_bytes / 2) / wk.seg_bytes;
-            seg_rows = (u.rows + nseg - 1) / nseg;
+    const uint32_t nC = gridDim.x;
+    for (; cur.ui < wk.U; ++cur.ui, cur.seg_item = 0, cur.tail_done = false) {
+        if (st) {
+            j.op = st->op[cur.ui];
+            if (j.op == OP_NONE)
+                continue;
+            j.u = st->u[cur.ui];
+        } else {
+            j.op = unit_op(wk, cur.ui);
+            if (recover ? (j.op != OP_RECOVER) : (j.op != OP_COMPRESS && j.op != OP_STATS))
+                continue;
+            j.u = wk.units ? wk.units[cur.ui] : wk.single;
+            const bool scaled = j.u.fmt != HILORE_FMT_E4M3FN_RAW;
+            if ((j.op == OP_COMPRESS && (!j.u.x || !j.u.codes || (scaled && !j.u.scales))) ||
+                (j.op == OP_STATS && (!j.u.x || !j.u.row_rms)) || (j.op == OP_RECOVER && (!j.u.out || !j.u.codes || (scaled && !j.u.scales))))
+                continue; // the unit lacks a buffer this operation needs: leave it untouched
+            if (j.op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
+                j.u.row_rms = nullptr; // token magnitudes were collected at capture time
         }
-        seg_rows = max((int64_t)gridDim.x, seg_rows);
-        while (cur.seg_row < u.rows) {
-            const int64_t s0 = cur.seg_row, n = min(seg_rows, u.rows - s0);
-            cur.seg_row += n;
-            if (n < (1ll << 31)) { // share[0..1] = floor(c * 2^32 / nC), floor((c + 1) * 2^32 / nC)
-                j.r0 = s0 + (int64_t)(((uint64_t)n * share[0]) >> 32);
-                j.r1 = s0 + (int64_t)(((uint64_t)n * share[1]) >> 32);
+        const bool per_row = !recover && j.u.row_rms != nullptr;
+        const UnitPlan p = plan_unit(wk, j.u, per_row);
+        const int nb = (int)(j.u.cols >> 6);
+        while (cur.seg_item < p.items) {
+            const int64_t s0 = cur.seg_item, n = min(p.seg_items, p.items - s0);
+            cur.seg_item += n;
+            uint32_t c = blockIdx.x + cur.rot;
+            c = c >= nC ? c - nC : c;
+            cur.rot += wk.rot_step;
+            cur.rot = cur.rot >= nC ? cur.rot - nC : cur.rot;
+            int64_t i0, i1;
+            if (n < (1ll << 31)) {
+                i0 = s0 + (int64_t)(((uint64_t)n * share_multiplier(wk, c)) >> 32);
+                i1 = s0 + (int64_t)(((uint64_t)n * share_multiplier(wk, c + 1)) >> 32);
             } else {
-                j.r0 = s0 + (n * (int64_t)blockIdx.x) / gridDim.x;
-                j.r1 = s0 + (n * (int64_t)(blockIdx.x + 1)) / gridDim.x;
+                i0 = s0 + (n * (int64_t)c) / nC;
+                i1 = s0 + (n * (int64_t)(c + 1)) / nC;
             }
-            if (j.r0 < j.r1)
-                return true; // the cursor already points at the next segment
+            if (i0 >= i1)
+                continue;
+            j.r0 = i0;
+            j.r1 = i1;
+            if (p.flat) { // the unit as rows of 8192 contiguous elements
+                j.u.rows = p.items;
+                j.u.cols = j.u.ld = kFlatCols;
+                j.rows_per_batch = 32;
+            } else {
+                j.rows_per_batch = max(1, slots / max(1, nb));
+            }
+            return true; // the cursor already points at the next window
+        }
+        if (p.flat && p.tail_chunks > 0 && !cur.tail_done) { // the last, partial piece: one short row
+            cur.tail_done = true;
+            uint32_t c = blockIdx.x + cur.rot;
+            c = c >= nC ? c - nC : c;
+            if (c == 0) {
+                const int64_t done = p.items * kFlatCols; // elements in whole pieces
+                j.u.x = static_cast<const uint16_t *>(j.u.x) + done;
+                j.u.out = static_cast<uint16_t *>(j.u.out) + done;
+                j.u.codes += done;
+                j.u.scales += done >> 6;
+                j.u.rows = 1;
+                j.u.cols = j.u.ld = (int64_t)p.tail_chunks * 16;
+                j.r0 = 0;
+                j.r1 = 1;
+                j.rows_per_batch = 1;
+                return true;
+            }
         }
     }
     return false;
@@ -483,12 +525,11 @@ __device__ __forceinline__ void careful_pair_fixup(const uint16_t *xa, const uin
 template <int FMT, bool CODES, bool SUMS>
 __device__ __forceinline__ void compress_rows(const uint16_t *__restrict__ x, uint8_t *__restrict__ codes,
                                               float *__restrict__ scales, float *__restrict__ row_rms, int64_t cols,
-                                              int64_t ld, int64_t r0, int64_t r1, float *sm_blocksum, int prefetch,
-                                              const uint32_t *tab)
+                                              int64_t ld, int64_t r0, int64_t r1, int rows_per_batch, float *sm_blocksum,
+                                              int prefetch, const uint32_t *tab)
 {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, q = lane & 3;
     const uint32_t nb = (uint32_t)(cols >> 6), cpr = (uint32_t)(cols >> 4);
-    const int rows_per_batch = max(1, kBlockSumSlots / (int)nb);
     const uint32_t magic = (uint32_t)((0x100000000ull + cpr - 1) / cpr); // chunk index (< 2^16) / cpr, exactly
     const float inv_cols = 1.0f / (float)cols;
     const bool contig = ld == cols;

@@ -15,7 +15,7 @@
 namespace hilore {
 
 constexpr int kCodecThreads = 256;   // 8 warps per CTA in the streaming codec kernels
-constexpr int kBlockSumSlots = 4096; // per-CTA shared slots for per-block sums of squares (16 KB)
+constexpr int kBlockSumSlots = 6144; // per-CTA shared slots for per-block sums of squares (24 KB)
 
 // ---- 256-bit global accesses (sm_100: one instruction moves 32 bytes per lane) ----
 __device__ __forceinline__ void ld_global_256(const void *p, uint32_t (&w)[8])

@@ -90,10 +90,9 @@ def test_7B_shaped_mixed_plan():
     x = [synth.activation_unit_device(gen, r, c, dev) for r, c in shapes]
     codes = [torch.full((r, c), 0xA5, dtype=torch.uint8, device=dev) for r, c in shapes]
     scales = [torch.full((r, c // 64), -7.0, dtype=torch.float32, device=dev) for r, c in shapes]
-    out = [torch.full((r, c), -3.0, dtype=torch.bfloat16, device=dev) if c < 10000 else None for r, c in shapes]
-    big_out = torch.full((rows, 18944), -3.0, dtype=torch.bfloat16, device=dev)   # shared by the wide units (memory)
+    out = [torch.full((r, c), -3.0, dtype=torch.bfloat16, device=dev) for r, c in shapes]   # no two units share a buffer
     rms = torch.full((U, rows), -1.0, dtype=torch.float32, device=dev)
-    units = [dict(x=x[i], codes=codes[i], scales=scales[i], out=out[i] if out[i] is not None else big_out,
+    units = [dict(x=x[i], codes=codes[i], scales=scales[i], out=out[i],
                   row_rms=rms[i], rows=r, cols=c, fmt=api.FMT_E4M3FN_BLK, block=64) for i, (r, c) in enumerate(shapes)]
     udev, uhost = api.make_unit_table(units, dev)
     avail = torch.full((U,), H, dtype=torch.uint8, device=dev)
@@ -154,16 +153,12 @@ def test_7B_shaped_mixed_plan():
     for u in narrow_L[:3] + narrow_L[-2:]:
         check_rows(x[u], codes[u], scales[u], out[u], rms[u], sample_rows(rng, rows, 12), api.FMT_E4M3FN_BLK)
     for u in wide_L[:2] + wide_L[-1:]:
-        check_rows(x[u], codes[u], scales[u], None, rms[u], sample_rows(rng, rows, 8), api.FMT_E4M3FN_BLK, what=("codes", "rms"))
-    if wide_L:   # the shared reconstruction buffer holds the last wide L unit
-        u = wide_L[-1]
-        check_rows(x[u], codes[u], scales[u], big_out, rms[u], sample_rows(rng, rows, 8), api.FMT_E4M3FN_BLK)
+        check_rows(x[u], codes[u], scales[u], out[u], rms[u], sample_rows(rng, rows, 8), api.FMT_E4M3FN_BLK)
     for u in [v for v in range(U) if a[v] != L][:8]:          # H keeps its bundle, R is recomputed: nothing written
         assert bool((codes[u] == 0xA5).all()) and bool((scales[u] == -7.0).all())
-        if out[u] is not None:
-            assert bool((out[u] == -3.0).all())
+        assert bool((out[u] == -3.0).all())
         check_rows(x[u], None, None, None, rms[u], sample_rows(rng, rows, 6), api.FMT_E4M3FN_BLK, what=("rms",))
-    del x, codes, scales, out, big_out
+    del x, codes, scales, out
     torch.cuda.empty_cache()
 
 
