@@ -217,3 +217,156 @@ def test_4GiB_unit_uses_64_bit_offsets():
         assert bool((codes[3 * base.shape[0]: 4 * base.shape[0]] == first).all())
         del codes, scales, rms, out
         torch.cuda.empty_cache()
+
+
+def xor_fold(t: torch.Tensor) -> int:
+    """xor of all 64-bit words of a device tensor (its byte size must be a multiple of 8)."""
+    w = t.contiguous().view(torch.uint8).view(-1).view(torch.int64)
+    while w.numel() > 1:
+        h = w.numel() // 2
+        rest = w[2 * h:]
+        w = torch.bitwise_xor(w[:h], w[h:2 * h])
+        if rest.numel():
+            w = torch.cat([w, rest])
+    return int(w.item())
+
+
+def xor_fold_host(a: np.ndarray) -> int:
+    return int(np.bitwise_xor.reduce(np.ascontiguousarray(a).view(np.int64).reshape(-1)))
+
+
+def oracle_unit(xb: np.ndarray, threads=16):
+    """Codes, scales, reconstruction and token RMS of a whole unit from the oracle, its C calls spread over row ranges."""
+    from concurrent.futures import ThreadPoolExecutor
+    cuts = [xb.shape[0] * i // threads for i in range(threads + 1)]
+
+    def part(ab):
+        x = xb[ab[0]:ab[1]]
+        c, s = oracle.compress(x, oracle.FMT_E4M3FN_BLK, 64)
+        return c, s, oracle.recover(c, s, oracle.FMT_E4M3FN_BLK, 64), oracle.row_rms(x)
+    with ThreadPoolExecutor(threads) as pool:
+        parts = list(pool.map(part, zip(cuts[:-1], cuts[1:])))
+    return tuple(np.concatenate([p[i] for p in parts]) for i in range(4))
+
+
+def test_1p5B_shaped_whole_units_and_checksums_over_microbatches():
+    """configs[1]: the step bench.py's 1.5B-shaped leg times, on fresh activations per microbatch.  Microbatches 0 and
+    63: one narrow and one wide unit compared WHOLE with the oracle (codes, scale bits, reconstruction, token RMS), and
+    their xor-folds with the oracle's.  Eight microbatches: xor-fold of the codes and scale bits of all 84 units,
+    equal between two runs on the same inputs (same bits whatever the scheduling) and different between microbatches."""
+    dev = torch.device("cuda", 0)
+    cfg = bench.CONFIGS[2]
+    wl = bench.Workload(api, synth, cfg, seed=0, device=dev)
+    mbs = [0, 9, 18, 27, 36, 45, 54, 63]
+
+    def run(mb, check_whole):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(1000 + mb)
+        for i, (r, c) in enumerate(wl.shapes):
+            wl.x[i].copy_(synth.activation_unit_device(gen, r, c, dev))
+        for t in wl.codes + wl.scales:
+            t.fill_(0)
+        wl.step(mb)
+        torch.cuda.synchronize()
+        sums = [(xor_fold(wl.codes[u]), xor_fold(wl.scales[u])) for u in range(wl.U)]
+        if check_whole:
+            for u in (3 * (mb % 28), 3 * (mb % 28) + 2):         # a narrow and a wide unit of one layer
+                oc, osc, oout, orms = oracle_unit(bits(wl.x[u]))
+                assert np.array_equal(wl.codes[u].cpu().numpy(), oc)
+                assert np.array_equal(wl.scales[u].cpu().numpy().view(np.uint32), osc.view(np.uint32))
+                assert np.array_equal(bits(wl.out[u]), oout)
+                assert G.rel_err(wl.rms[u].cpu().numpy(), orms).max() <= 1e-5
+                assert sums[u] == (xor_fold_host(oc), xor_fold_host(osc))
+        return sums
+
+    first = {mb: run(mb, mb in (0, 63)) for mb in mbs}
+    again = {mb: run(mb, False) for mb in mbs}
+    assert first == again
+    assert len({tuple(v) for v in first.values()}) == len(mbs)
+    del wl
+    torch.cuda.empty_cache()
+
+
+def test_7B_shaped_plan_with_demoted_candidates():
+    """configs[2], second run: a quarter of the units captured as L candidates, a quarter as R candidates, the rest H,
+    through CAPTURE / DECIDE / ENCODE / RECOVER at full size.  Desired actions outside a unit's candidate set are
+    demoted to R; R candidates are never touched; H candidates assigned L are encoded after the forward pass."""
+    dev = torch.device("cuda", 0)
+    rows, layers = 16384, 28
+    shapes = synth.layer_unit_shapes("7B", rows, layers)
+    U = len(shapes)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(11)
+    x = [synth.activation_unit_device(gen, r, c, dev) for r, c in shapes]
+    codes = [torch.full((r, c), 0xA5, dtype=torch.uint8, device=dev) for r, c in shapes]
+    scales = [torch.full((r, c // 64), -7.0, dtype=torch.float32, device=dev) for r, c in shapes]
+    out = [torch.full((r, c), -3.0, dtype=torch.bfloat16, device=dev) for r, c in shapes]
+    rms = torch.full((U, rows), -1.0, dtype=torch.float32, device=dev)
+    units = [dict(x=x[i], codes=codes[i], scales=scales[i], out=out[i], row_rms=rms[i], rows=r, cols=c,
+                  fmt=api.FMT_E4M3FN_BLK, block=64) for i, (r, c) in enumerate(shapes)]
+    udev, uhost = api.make_unit_table(units, dev)
+    q = np.array([(L, H, R, H)[i % 4] for i in range(U)], dtype=np.uint8)     # 21 L, 21 R, 42 H, every width in each
+    assert [(q == v).sum() for v in (L, R, H)] == [21, 21, 42]
+    avail = torch.from_numpy(q).to(dev)
+    action = torch.zeros(U, dtype=torch.uint8, device=dev)
+    rec = torch.zeros(U, dtype=torch.uint8, device=dev)
+    retained = torch.zeros(U, dtype=torch.int64, device=dev)
+    psi = torch.zeros(U, dtype=torch.float32, device=dev)
+    expo = torch.zeros(U, dtype=torch.float32, device=dev)
+    call = lambda phase, **k: api.hilore_plan_apply(udev, uhost, U, phase, k.get("E"), k.get("kappa"), k.get("ebar"),
+                                                    k.get("lo", 0.0), k.get("hi", 0.0), avail, action, k.get("psi"), rec,
+                                                    retained)
+    call(api.PHASE_CAPTURE)
+    torch.cuda.synchronize()
+    rms_h = rms.cpu().numpy()
+    for u in range(U):                                      # R candidates: nothing written; H: token RMS only
+        if q[u] == R:
+            assert np.all(rms_h[u] == -1.0) and bool((codes[u][::4097] == 0xA5).all())
+        elif q[u] == H:
+            assert np.all(rms_h[u] > 0) and bool((codes[u] == 0xA5).all()) and bool((scales[u] == -7.0).all())
+        else:
+            assert np.all(rms_h[u] > 0) and not bool((scales[u] == -7.0).any())
+    ro = synth.rollout(12, 16, 16, 2048)
+    mb, n_mb = 3, 8
+    sl = slice(mb * n_mb, (mb + 1) * n_mb)
+    t = lambda a: torch.from_numpy(a).to(dev)
+    omega = torch.empty((n_mb, 2048), dtype=torch.float32, device=dev)
+    nws = api.hilore_workspace_bytes(U, rows)
+    ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+    rms.clamp_(min=0.0)                                     # R candidates have no token RMS: a defined value for the score
+    api.hilore_coeffs_exposure(t(ro.rewards), ro.n_resp, 16, mb * n_mb, n_mb, 2048, t(ro.logp_new[sl]), t(ro.logp_old[sl]),
+                               None, t(ro.mask[sl]), ro.n_valid, None, 0.2, 0.0, 1e-6, rms, U, rows, 0, 1e-8, omega, expo,
+                               None, ws, nws)
+    kappa = np.random.default_rng(13).uniform(0.5, 2.0, U).astype(np.float32)
+    ebar = np.full(U, 0.0266, dtype=np.float32)
+    E = expo.cpu().numpy()
+    psi_h = (kappa * E).astype(np.float32) * ebar
+    live = np.sort(psi_h[q != R])
+    lo, hi = float((live[30] + live[31]) / 2), float((live[44] + live[45]) / 2)
+    call(api.PHASE_DECIDE, E=expo, kappa=t(kappa), ebar=t(ebar), lo=lo, hi=hi, psi=psi)
+    a = action.cpu().numpy()
+    # the plan from the oracle on the same exposure bits (a unit's action depends on its own psi only)
+    oa, opsi, orec, oret = oracle.plan(E, kappa, ebar, lo, hi, q, [s[0] for s in shapes], [s[1] for s in shapes], [1] * U, [64] * U)
+    assert np.array_equal(a, oa) and np.array_equal(rec.cpu().numpy(), orec)
+    assert np.array_equal(psi.cpu().numpy().view(np.uint32), opsi.view(np.uint32))
+    assert np.array_equal(retained.cpu().numpy().view(np.uint64), oret)
+    assert np.all(a[q == R] == R) and np.all(a[(q == L)] != H)                 # demotion
+    assert ((q == L) & (a == R)).sum() > 0 and ((q == H) & (a == L)).sum() > 0  # both kinds occur in this draw
+    codes_before = {u: xor_fold(codes[u]) for u in range(U) if q[u] == L}
+    call(api.PHASE_ENCODE)
+    call(api.PHASE_RECOVER)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(14)
+    enc = [u for u in range(U) if q[u] == H and a[u] == L]
+    cap = [u for u in range(U) if q[u] == L and a[u] == L]
+    for u in enc[:3] + enc[-2:] + cap[:2] + cap[-1:]:
+        check_rows(x[u], codes[u], scales[u], out[u], rms[u], sample_rows(rng, rows, 10), api.FMT_E4M3FN_BLK)
+    for u in codes_before:                                   # ENCODE leaves the units captured as L alone
+        assert xor_fold(codes[u]) == codes_before[u]
+    for u in range(U):
+        if a[u] != L:                                       # nothing decoded into units that are not L
+            assert bool((out[u][::257] == -3.0).all())
+        if q[u] == R or (q[u] == H and a[u] != L):          # never compressed
+            assert bool((codes[u] == 0xA5).all()) and bool((scales[u] == -7.0).all())
+    del x, codes, scales, out
+    torch.cuda.empty_cache()

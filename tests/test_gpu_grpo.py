@@ -1,12 +1,15 @@
 """Parity of hilore_mask_count / hilore_grpo_coeffs / hilore_unit_exposure with the CPU oracle.
 
 fp32 outputs: 1e-5 relative (signed zeros equal).  The clip indicator is an integer decided by an
-fp32 compare of r = exp(s - s_old); the oracle rounds a double exp, the kernel uses expf, so a slot
-whose oracle ratio lies within 4 ulp of a clip bound may legitimately differ and is excused (and
+fp32 compare of r = exp(s - s_old); the oracle rounds a double exp, the kernel evaluates
+ex2.approx(d * log2 e), whose relative error is bounded by |d| * 2^-24 + 2^-22 (2.4e-7 plus 6e-8 per
+unit of |d|: about 3 ulp of a ratio near the clip bounds 0.8 and 1.2, and below 6e-6 up to |d| = 80), so
+a slot whose oracle ratio lies within 4 ulp of a clip bound may legitimately differ and is excused (and
 counted).  All calls go through the C ABI.
 """
 import numpy as np
 import pytest
+import torch
 
 import oracle
 from paper_2609_33570_b200 import api, synth
@@ -241,3 +244,60 @@ def test_k3_term_alone_over_a_wide_range_of_log_ratios():
     assert np.all(adv == 0)
     w, _, _ = oracle.grpo_coeffs(adv, ro.logp_new, ro.logp_old, ro.logp_ref, ro.mask, N_norm=ro.n_valid, beta=0.25)
     assert G.rel_err(got["omega"], w).max() <= RTOL
+
+
+def test_normaliser_of_this_call_matches_the_oracles_zero_rule():
+    """The oracle takes N_norm = 0 as "the sum of the mask over this call".  The library keeps no scratch of its own,
+    so the same rule is two stream-ordered calls: hilore_mask_count of the call's mask into a device word, which the
+    coefficient kernel reads (no host synchronisation); a host N_norm <= 0 without that word is refused."""
+    ro = synth.rollout(51, 4, 8, 512, rewards="uniform", lengths="uniform")
+    off, n_rows = 8, 16
+    sl = slice(off, off + n_rows)
+    R, ln, lo, mk = G.dev(ro.rewards), G.dev(ro.logp_new[sl]), G.dev(ro.logp_old[sl]), G.dev(ro.mask[sl])
+    omega = G.Guarded(n_rows * ro.T * 4)
+    for bad in (0, -5):
+        st = api.hilore_grpo_coeffs(R, ro.n_resp, ro.G, off, n_rows, ro.T, ln, lo, None, mk, bad, None, 0.2, 0.0, 1e-6, None,
+                                    omega.ptr(), None, None, check=False)
+        assert st == api.ZERO_NORM
+    ndev = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+    api.hilore_mask_count(mk, mk.numel(), ndev)
+    api.hilore_grpo_coeffs(R, ro.n_resp, ro.G, off, n_rows, ro.T, ln, lo, None, mk, 0, ndev, 0.2, 0.0, 1e-6, None, omega.ptr(),
+                           None, None)
+    got = omega.numpy(np.float32, (n_rows, ro.T))
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, r, _ = oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=0)
+    assert int(ndev.item()) == int(ro.mask[sl].sum())
+    hi, lo_b = np.float32(1.2), np.float32(0.8)
+    near = (np.abs(r - hi) <= 4 * np.spacing(hi)) | (np.abs(r - lo_b) <= 4 * np.spacing(lo_b))
+    assert G.rel_err(got[~near], w[~near]).max() <= RTOL
+    # a call whose mask is empty: the oracle refuses (no normaliser), the device word is 0 and every coefficient is 0
+    empty = np.zeros_like(ro.mask[sl])
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, empty, N_norm=0)
+    assert e.value.status == oracle.ZERO_NORM
+    mk0 = G.dev(empty)
+    api.hilore_mask_count(mk0, mk0.numel(), ndev)
+    api.hilore_grpo_coeffs(R, ro.n_resp, ro.G, off, n_rows, ro.T, ln, lo, None, mk0, 0, ndev, 0.2, 0.0, 1e-6, None, omega.ptr(),
+                           None, None)
+    assert int(ndev.item()) == 0 and np.all(omega.numpy(np.float32, (n_rows, ro.T)) == 0)
+
+
+def test_coefficients_at_the_top_of_the_sweep_on_sampled_responses():
+    """2^24 slots at G = 16, T = 1024 (16 384 responses, the largest point of the bandwidth sweep), with and without
+    the K3 term: the responses of a sample of prompt groups against the oracle, element by element."""
+    ro = synth.rollout(61, 1024, 16, 1024)
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    rng = np.random.default_rng(7)
+    groups = sorted(set([0, 1, 511, 512, 1022, 1023] + rng.integers(0, 1024, 10).tolist()))
+    rows = np.concatenate([np.arange(g * 16, g * 16 + 16) for g in groups])
+    R, ln, lo, lr, mk = (G.dev(a) for a in (ro.rewards, ro.logp_new, ro.logp_old, ro.logp_ref, ro.mask))
+    for beta in (0.0, 1e-3):
+        omega = torch.full((ro.n_resp, ro.T), 7.0, dtype=torch.float32, device="cuda")
+        a_out = torch.full((ro.n_resp,), 7.0, dtype=torch.float32, device="cuda")
+        api.hilore_grpo_coeffs(R, ro.n_resp, ro.G, 0, ro.n_resp, ro.T, ln, lo, lr if beta else None, mk, ro.n_valid, None, 0.2,
+                               beta, 1e-6, a_out, omega, None, None)
+        got = dict(adv=a_out.cpu().numpy()[rows], omega=omega.cpu().numpy()[rows])
+        sub = synth.Rollout(len(groups), 16, ro.T, ro.rewards[rows], ro.logp_new[rows], ro.logp_old[rows], ro.logp_ref[rows],
+                            ro.mask[rows], ro.lengths[rows])
+        check_coeffs(sub, got, N=ro.n_valid, beta=beta)
+        assert not bool((omega == 7.0).any()) and not bool((a_out == 7.0).any())      # every slot and response written

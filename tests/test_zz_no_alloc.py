@@ -1,11 +1,13 @@
 """hilore_unit_exposure_static: the exposure reduction for callers that may not allocate (its partial
 sums live in a fixed array inside the library).  Checked against hilore_unit_exposure, which takes the
-scratch from the caller, on two calls in a row -- the second call finds the first call's partial sums
-still in the shared array and must not be disturbed by them.  Collected last on purpose."""
+scratch from the caller, and against the CPU oracle, on two calls in a row -- the second call finds the
+first call's partial sums still in the shared array and must not be disturbed by them.  Collected last
+on purpose."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2609_33570_b200 import api, synth
 from tests import gpu_util as G
 
@@ -38,6 +40,8 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
         got_E, got_sw = _static(omega, mask, rms)
         assert G.rel_err(got_E, want_E).max() <= RTOL
         assert abs(got_sw - want_sw) <= RTOL * abs(want_sw)
+        oE, osw = oracle.unit_exposure(omega, mask, rms)       # and both against the oracle's definition
+        assert G.rel_err(got_E, oE).max() <= RTOL and abs(got_sw - osw) <= RTOL * abs(osw)
     # the scalar path (row_shift = 1) goes through the same array
     omega, mask, rms = small
     mask = mask.copy()
@@ -45,6 +49,7 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
     want_E, _ = G.unit_exposure(omega, mask, rms, row_shift=1)
     got_E, _ = _static(omega, mask, rms, row_shift=1)
     assert G.rel_err(got_E, want_E).max() <= RTOL
+    assert G.rel_err(got_E, oracle.unit_exposure(omega, mask, rms, row_shift=1)[0]).max() <= RTOL
 
 
 def test_static_scratch_rejects_problems_beyond_its_size():
