@@ -225,7 +225,7 @@ class Workload:
         self.kappa = torch.from_numpy(kgen.uniform(0.5, 2.0, U).astype(np.float32)).to(device)
         self.ebar = torch.full((U,), 0.025, dtype=torch.float32, device=device)
         self.omega = torch.empty((self.mb_resp, T), dtype=torch.float32, device=device)
-        self.ws_bytes = api.hilore_workspace_bytes(U, self.rows)
+        self.ws_bytes = api.hilore_scores_plan_workspace_bytes(U, self.rows)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device=device)
         self.n_valid = ro.n_valid
         self.elements = sum(r * c for r, c in self.shapes)
@@ -240,14 +240,14 @@ class Workload:
             self.bytes_encode = [0] * self.n_plan
             self.bytes_recover = [0] * self.n_plan
             self.expected_action = [None] * self.n_plan
-            self.launches_per_step = 6   # capture, scores (2), decide, encode, recover
+            self.launches_per_step = 4   # capture, scores + plan, encode, recover (and one 4-byte memset)
         else:
             self.bytes_capture = sum(codec_bytes(r, c, True, True) for r, c in self.shapes)
             self.n_plan = self.n_microbatches
             self.tau = [(inf, inf)] * self.n_plan
             self.bytes_encode = [0] * self.n_plan
             self.bytes_recover = [sum(codec_bytes(r, c, True, False) for r, c in self.shapes)] * self.n_plan
-            self.launches_per_step = 5   # capture, scores (2), decide, recover
+            self.launches_per_step = 3   # capture, scores + plan, recover (and one 4-byte memset)
 
     def bytes_step(self, mb):
         mb %= self.n_plan
@@ -266,6 +266,14 @@ class Workload:
         a.hilore_coeffs_exposure(self.rewards, self.n_resp, self.G, mb * self.mb_resp, self.mb_resp, self.T, self.logp_new[sl],
                                  self.logp_old[sl], None, self.mask[sl], self.n_valid, None, 0.2, 0.0, 1e-6, self.rms,
                                  self.U, self.rows, 0, 1e-8, self.omega, self.exposure, None, self.ws, self.ws_bytes)
+
+    def scores_plan(self, mb, tau_lo, tau_hi):
+        a = self.api
+        sl = slice(mb * self.mb_resp, (mb + 1) * self.mb_resp)
+        a.hilore_scores_plan(self.rewards, self.n_resp, self.G, mb * self.mb_resp, self.mb_resp, self.T, self.logp_new[sl],
+                             self.logp_old[sl], None, self.mask[sl], self.n_valid, None, 0.2, 0.0, 1e-6, self.rms, self.U,
+                             self.rows, 0, 1e-8, self.omega, self.exposure, None, self.units_dev, self.kappa, self.ebar, tau_lo,
+                             tau_hi, self.avail, self.action, self.psi, self.recompute, self.retained, self.ws, self.ws_bytes)
 
     def decide(self, tau_lo, tau_hi):
         a = self.api
@@ -319,9 +327,8 @@ class Workload:
         rec("capture", 0)
         self.capture()
         rec("capture", 1)
-        rec("scores", 0)   # coefficients and their reduction to exposure scores (one sweep), then the plan
-        self.scores(mb)
-        self.decide(*self.tau[mb])
+        rec("scores", 0)   # coefficients, their reduction to exposure scores and the plan: one launch
+        self.scores_plan(mb, *self.tau[mb])
         rec("scores", 1)
         if self.mixed:
             rec("encode", 0)
@@ -678,7 +685,7 @@ def main():
                             [(b_rec, kern_ms["recover"], DRAM_PER_ALGORITHMIC["recover"])])
     kernels["recover_L_units" if wl.mixed else "recover"] = {"ms": kern_ms["recover"], **fractions(b_rec / kern_ms["recover"] / 1e6, peak)}
     kernels["scores_decide_microbatch"] = {"us": kern_ms["scores"] * 1e3, "tokens_per_s": wl.rows / kern_ms["scores"] * 1e3,
-                                           "launches": 3}
+                                           "launches": 1}
     out = {
         "metric": METRIC, "value": world * bytes_timed / (ms_step * args.steps) / 1e6, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,

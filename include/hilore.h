@@ -67,6 +67,8 @@ enum {
     HILORE_PHASE_RECOVER = 3  /* backward-time recovery: units with action L are decoded to bf16         */
 };
 
+struct hilore_unit; /* one recovery unit of a microbatch; defined with hilore_plan_apply below */
+
 const char *hilore_status_string(int status);
 /* Version of this ABI (major * 1000 + minor). */
 int hilore_abi_version(void);
@@ -125,6 +127,32 @@ int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G
                            float adv_eps, const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
                            float eps_alpha, float *omega, float *exposure, float *sum_abs_omega, void *workspace,
                            size_t workspace_bytes, void *stream);
+
+/*
+ * The score refresh of one microbatch in ONE kernel launch: hilore_coeffs_exposure followed by
+ * hilore_plan_apply(HILORE_PHASE_DECIDE) (Algorithm 1, lines "coefficients", "exposure", risk score and allocation;
+ * Eqs. "update-coefficient", "mlp-weighted-exposure", "token-weighted-risk", "available-recovery-actions").  The CTA
+ * that finishes last among those of a group of eight units adds the group's per-tile partial sums in the fixed order
+ * of the two-kernel form and takes the plan decisions of its units, so omega, exposure, psi, action_io, recompute and retained_bytes are bit for bit those of
+ * the separate calls, whichever CTA that is.  Between forward and backward of a microbatch this is one launch (plus a
+ * 4-byte memset) instead of four.
+ *   Arguments as in hilore_coeffs_exposure (omega REQUIRED, U > 0, n_rows * T > 0) and in the DECIDE phase of
+ *   hilore_plan_apply (units_dev, kappa, ebar, avail, action_io REQUIRED; psi, recompute, retained_bytes opt; the
+ *   unit table is only read for rows, cols and fmt, on the device).
+ *   workspace   at least hilore_scores_plan_workspace_bytes(U, n_rows * T) bytes, 16-byte aligned: the partial sums
+ *               and, behind them, the counters of finished CTAs, which the call sets to zero itself.
+ *   Microbatches beyond the one-sweep form's limits (see hilore_coeffs_exposure) run the coefficient pass first and
+ *   then the reduction + plan launch.
+ */
+int hilore_scores_plan(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset, int64_t n_rows,
+                       int64_t T, const float *logp_new, const float *logp_old, const float *logp_ref,
+                       const uint8_t *mask, int64_t N_norm, const int64_t *N_norm_dev, float clip_eps, float beta,
+                       float adv_eps, const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                       float eps_alpha, float *omega, float *exposure, float *sum_abs_omega,
+                       const struct hilore_unit *units_dev, const float *kappa, const float *ebar, float tau_lo,
+                       float tau_hi, const uint8_t *avail, uint8_t *action_io, float *psi, uint8_t *recompute,
+                       uint64_t *retained_bytes, void *workspace, size_t workspace_bytes, void *stream);
+size_t hilore_scores_plan_workspace_bytes(int32_t U, int64_t n_tok);
 
 /*
  * The coefficient and exposure passes on the packed (padding-removed) layout of the paper's DSR-sub execution

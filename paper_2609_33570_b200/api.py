@@ -28,7 +28,7 @@ EXPORTS = ("hilore_status_string", "hilore_abi_version", "hilore_mask_count", "h
            "hilore_relative_error", "hilore_relative_error_workspace_bytes", "hilore_fit_kappa",
            "hilore_grpo_coeffs_variant", "hilore_omega_diagnostics", "hilore_omega_diagnostics_workspace_bytes",
            "hilore_grpo_coeffs_packed", "hilore_unit_exposure_packed", "hilore_codec_relative_error",
-           "hilore_coeffs_exposure")
+           "hilore_coeffs_exposure", "hilore_scores_plan", "hilore_scores_plan_workspace_bytes")
 
 
 class HiloreUnit(C.Structure):
@@ -90,6 +90,10 @@ def lib() -> C.CDLL:
         _lib.hilore_unit_exposure_packed.argtypes = [vp, vp, i64, vp, i64, vp, i32, i64, i32, f32, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_coeffs_exposure.argtypes = [vp, i64, i32, i64, i64, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32, vp, i32, i64,
                                                 i32, f32, vp, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_scores_plan.argtypes = [vp, i64, i32, i64, i64, i64, vp, vp, vp, vp, i64, vp, f32, f32, f32, vp, i32, i64, i32,
+                                            f32, vp, vp, vp, vp, vp, vp, f32, f32, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]
+        _lib.hilore_scores_plan_workspace_bytes.restype = C.c_size_t
+        _lib.hilore_scores_plan_workspace_bytes.argtypes = [i32, i64]
         _lib.hilore_codec_relative_error.argtypes = [vp, i64, i64, i64, i32, i32, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_omega_diagnostics.argtypes = [vp, vp, vp, vp, i64, i64, f32, vp, vp, vp, vp, C.c_size_t, vp]
         _lib.hilore_omega_diagnostics_workspace_bytes.restype = C.c_size_t
@@ -101,7 +105,7 @@ def lib() -> C.CDLL:
             if name not in ("hilore_status_string", "hilore_workspace_bytes", "hilore_static_scratch_bytes",
                             "hilore_allocate_workspace_bytes", "hilore_risk_budget",
                             "hilore_relative_error_workspace_bytes", "hilore_fit_kappa",
-                            "hilore_omega_diagnostics_workspace_bytes"):
+                            "hilore_omega_diagnostics_workspace_bytes", "hilore_scores_plan_workspace_bytes"):
                 getattr(_lib, name).restype = C.c_int
     return _lib
 
@@ -181,6 +185,22 @@ def hilore_coeffs_exposure(rewards, n_resp_total, G, resp_offset, n_rows, T, log
                                       _ptr(row_rms), U, rms_ld, row_shift, eps_alpha, _ptr(omega), _ptr(exposure),
                                       _ptr(sum_abs_omega), _ptr(workspace), workspace_bytes, _stream(stream))
     return _check(st, "hilore_coeffs_exposure", check)
+
+
+def hilore_scores_plan_workspace_bytes(U, n_tok):
+    return int(lib().hilore_scores_plan_workspace_bytes(U, n_tok))
+
+
+def hilore_scores_plan(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask, N_norm, N_norm_dev,
+                       clip_eps, beta, adv_eps, row_rms, U, rms_ld, row_shift, eps_alpha, omega, exposure, sum_abs_omega,
+                       units_dev, kappa, ebar, tau_lo, tau_hi, avail, action_io, psi, recompute, retained_bytes, workspace,
+                       workspace_bytes, stream=None, check=True):
+    st = lib().hilore_scores_plan(_ptr(rewards), n_resp_total, G, resp_offset, n_rows, T, _ptr(logp_new), _ptr(logp_old),
+                                  _ptr(logp_ref), _ptr(mask), N_norm, _ptr(N_norm_dev), clip_eps, beta, adv_eps, _ptr(row_rms), U,
+                                  rms_ld, row_shift, eps_alpha, _ptr(omega), _ptr(exposure), _ptr(sum_abs_omega), _ptr(units_dev),
+                                  _ptr(kappa), _ptr(ebar), tau_lo, tau_hi, _ptr(avail), _ptr(action_io), _ptr(psi),
+                                  _ptr(recompute), _ptr(retained_bytes), _ptr(workspace), workspace_bytes, _stream(stream))
+    return _check(st, "hilore_scores_plan", check)
 
 
 def hilore_codec_relative_error(x, rows, cols, ld, fmt, block, e_out, norms2, workspace, workspace_bytes, stream=None,

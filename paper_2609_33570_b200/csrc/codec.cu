@@ -81,30 +81,12 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_k
 }
 
 // psi, threshold rule, availability demotion, recompute flags and retained bytes for U units.
-__global__ void plan_decide_kernel(const hilore_unit *units, int U, const float *exposure, const float *kappa,
-                                   const float *ebar, float tau_lo, float tau_hi, const uint8_t *avail,
-                                   uint8_t *action_io, float *psi, uint8_t *recompute, uint64_t *retained_bytes)
+__global__ void plan_decide_kernel(PlanTail p, int U, const float *exposure)
 {
-    for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x) {
-        uint32_t want = action_io[u];
-        if (exposure != nullptr) {
-            const float p = __fmul_rn(__fmul_rn(kappa[u], exposure[u]), ebar[u]);
-            if (psi) psi[u] = p;
-            want = (p < tau_lo) ? HILORE_ACT_L : ((p >= tau_hi) ? HILORE_ACT_H : HILORE_ACT_R);
-        }
-        const uint32_t q = avail[u];
-        const bool ok = (q == HILORE_ACT_H) || (q == HILORE_ACT_L && want != HILORE_ACT_H) || (want == HILORE_ACT_R);
-        uint32_t a = (ok && want <= HILORE_ACT_L) ? want : (uint32_t)HILORE_ACT_R;
-        action_io[u] = (uint8_t)a;
-        if (recompute) recompute[u] = (a == HILORE_ACT_R);
-        if (retained_bytes) {
-            const uint64_t n = (uint64_t)units[u].rows * (uint64_t)units[u].cols;
-            uint64_t b = 0;
-            if (a == HILORE_ACT_H) b = 2 * n;
-            else if (a == HILORE_ACT_L) b = n + (units[u].fmt == HILORE_FMT_E4M3FN_RAW ? 0 : 4 * (n / HILORE_BLOCK));
-            retained_bytes[u] = b;
-        }
-    }
+    grid_dependency_wait();
+    grid_dependency_release();
+    for (int u = blockIdx.x * blockDim.x + threadIdx.x; u < U; u += gridDim.x * blockDim.x)
+        decide_unit(p, u, exposure ? exposure + u : nullptr);
 }
 
 // Host-side validation of one unit descriptor.  `strict` (single-unit entry points): the buffers the
@@ -279,8 +261,19 @@ extern "C" int hilore_plan_apply(const hilore_unit *units_dev, const hilore_unit
     if (phase == HILORE_PHASE_DECIDE) {
         if (exposure != nullptr && (kappa == nullptr || ebar == nullptr))
             return HILORE_INVALID_ARG;
-        plan_decide_kernel<<<1, 128, 0, st>>>(units_dev, U, exposure, kappa, ebar, tau_lo, tau_hi, avail, action_io,
-                                              psi, recompute, retained_bytes);
+        PlanTail p{};
+        p.units = units_dev;
+        p.kappa = kappa;
+        p.ebar = ebar;
+        p.tau_lo = tau_lo;
+        p.tau_hi = tau_hi;
+        p.avail = avail;
+        p.action_io = action_io;
+        p.psi = psi;
+        p.recompute = recompute;
+        p.retained_bytes = retained_bytes;
+        if (launch_dependent(plan_decide_kernel, dim3(1), dim3(128), 0, st, p, (int)U, exposure) != cudaSuccess)
+            return HILORE_CUDA;
         return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
     }
     // one launch per slice of at most kStageUnits units (the kernels stage a slice's descriptors in shared memory)

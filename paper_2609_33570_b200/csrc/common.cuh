@@ -193,6 +193,62 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may become resident while the previous
+// kernel of the stream drains.  Every kernel launched this way executes griddepcontrol.wait before its first
+// access to global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// Risk score and H / L / R gating of one unit (Eq. "token-weighted-risk", Eq. "available-recovery-actions"; the
+// threshold rule stands in for the paper's allocator): psi = fl32(fl32(kappa E) ebar); desired = L below tau_lo, H
+// from tau_hi on, else R (NaN -> R); outside the candidate set of q -> R.  `E` == nullptr: the desired action is
+// action_io[u] as given.
+struct PlanTail {
+    const hilore_unit *units;
+    const float *kappa, *ebar;
+    float tau_lo, tau_hi;
+    const uint8_t *avail;
+    uint8_t *action_io;
+    float *psi;
+    uint8_t *recompute;
+    uint64_t *retained_bytes;
+};
+
+__device__ __forceinline__ void decide_unit(const PlanTail &p, int u, const float *E)
+{
+    uint32_t want = p.action_io[u];
+    if (E != nullptr) {
+        const float v = __fmul_rn(__fmul_rn(p.kappa[u], *E), p.ebar[u]);
+        if (p.psi) p.psi[u] = v;
+        want = (v < p.tau_lo) ? HILORE_ACT_L : ((v >= p.tau_hi) ? HILORE_ACT_H : HILORE_ACT_R);
+    }
+    const uint32_t q = p.avail[u];
+    const bool ok = (q == HILORE_ACT_H) || (q == HILORE_ACT_L && want != HILORE_ACT_H) || (want == HILORE_ACT_R);
+    const uint32_t a = (ok && want <= HILORE_ACT_L) ? want : (uint32_t)HILORE_ACT_R;
+    p.action_io[u] = (uint8_t)a;
+    if (p.recompute) p.recompute[u] = (a == HILORE_ACT_R);
+    if (p.retained_bytes) {
+        const uint64_t n = (uint64_t)p.units[u].rows * (uint64_t)p.units[u].cols;
+        uint64_t b = 0;
+        if (a == HILORE_ACT_H) b = 2 * n;
+        else if (a == HILORE_ACT_L) b = n + (p.units[u].fmt == HILORE_FMT_E4M3FN_RAW ? 0 : 4 * (n / HILORE_BLOCK));
+        p.retained_bytes[u] = b;
+    }
+}
+
 inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // Immutable properties of the devices, looked up once per device and process (no device memory involved).

@@ -548,6 +548,30 @@ constexpr int kExpThreads = 256;
 constexpr int kExpTile = kExpThreads * 4; // slots per CTA
 constexpr int kExpUnits = 8;              // units per CTA (omega and mask are read once for all of them)
 
+// One warp adds the per-tile partials of unit u in a fixed order and applies the closed form
+//   E_u = (S2_u + eps * S3) / (S1_u / |T_b| + eps),  S1 = sum a, S2 = sum |omega| a, S3 = sum |omega|.
+// Every lane returns E_u; *s3_out gets S3.
+__device__ __forceinline__ float exposure_of_unit(const double *part, int tok_row, int ntiles, int u, float eps_alpha, int lane,
+                                                  double *s3_out)
+{
+    double s1 = 0.0, s2 = 0.0, s3 = 0.0, cnt = 0.0;
+    for (int t = lane; t < ntiles; t += 32) { // tok_row: the row of partials that holds sum |omega| and |T_b|
+        s1 += __ldcg(part + ((int64_t)u * ntiles + t) * 2);
+        s2 += __ldcg(part + ((int64_t)u * ntiles + t) * 2 + 1);
+        s3 += __ldcg(part + ((int64_t)tok_row * ntiles + t) * 2);
+        cnt += __ldcg(part + ((int64_t)tok_row * ntiles + t) * 2 + 1);
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    s3 = warp_sum(s3);
+    cnt = warp_sum(cnt);
+    double E = 0.0;
+    if (cnt > 0.0)
+        E = (s2 + (double)eps_alpha * s3) / (s1 / cnt + (double)eps_alpha);
+    *s3_out = s3;
+    return (float)E;
+}
+
 // Inputs of the coefficient pass when it is fused into the exposure reduction (hilore_coeffs_exposure).
 constexpr int kFusedRows = 64; // responses one CTA's slots may span
 struct FusedCoeff {
@@ -575,6 +599,11 @@ struct ExpArgs {
     int n_seq;
     int steps;         // pieces of kExpTile slots per CTA
     FusedCoeff f;      // used by the fused kernel only
+    // single-launch form: the CTA that finishes last adds the partials and, if asked, takes the plan decisions
+    unsigned int *done; // counter of finished CTAs (zero before the launch), or nullptr: a second kernel finishes
+    float eps_alpha;
+    float *exposure, *sum_abs_omega;
+    PlanTail plan;      // plan.avail == nullptr: no decisions
 };
 
 // A CTA covers `steps` consecutive pieces of kExpTile slots for kExpUnits units: every thread accumulates its
@@ -597,6 +626,8 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
     const int tile = blockIdx.x;
     const int u0 = blockIdx.y * kExpUnits, nu = min(kExpUnits, a.U - u0);
     __shared__ double sm[kExpThreads / 32][2 * (kExpUnits + 1)];
+    grid_dependency_wait();
+    grid_dependency_release(); // the final reduction may become resident; it waits for this grid to complete
     __shared__ float s_A[FUSED ? kFusedRows : 1], s_coef[FUSED ? kFusedRows : 1];
     int64_t row_lo = 0;
     float f_kl = 0.0f, f_hi = 0.0f, f_lo = 0.0f;
@@ -623,7 +654,58 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
     float acc[2 * (kExpUnits + 1)];
 #pragma unroll
     for (int q = 0; q < 2 * (kExpUnits + 1); ++q) acc[q] = 0.0f;
-    for (int st = 0; st < a.steps; ++st) {
+    // Large token grids (the plain vector path): two pieces per trip, all their loads issued before the first
+    // use, so that a thread has twenty 16-byte loads in flight instead of ten; the sums are taken in the order of
+    // the one-piece loop below, whose results they equal bit for bit.
+    for (int st = 0; VEC && !FUSED && st < a.steps; st += 2) {
+        int64_t k[2];
+        bool ok[2];
+        uint32_t m[2] = {0, 0};
+        uint4 w[2], av[2][kExpUnits];
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            k[p] = ((int64_t)tile * a.steps + st + p) * kExpTile + (int64_t)tid * 4;
+            ok[p] = st + p < a.steps && k[p] < a.n_tok; // n_tok % 4 == 0: a group is valid as a whole
+            if (ok[p]) {
+                m[p] = __ldcs(reinterpret_cast<const unsigned int *>(a.mask + k[p]));
+                w[p] = ld_global_128_stream(a.omega + k[p]);
+#pragma unroll
+                for (int j = 0; j < kExpUnits; ++j)
+                    if (j < nu) av[p][j] = ld_global_128_stream(a.row_rms + (int64_t)(u0 + j) * a.rms_ld + k[p]);
+            }
+        }
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            if (!ok[p])
+                continue;
+            const float wv[4] = {__uint_as_float(w[p].x), __uint_as_float(w[p].y), __uint_as_float(w[p].z), __uint_as_float(w[p].w)};
+            bool mk[4];
+            float wabs[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                mk[i] = ((m[p] >> (8 * i)) & 0xFFu) != 0;
+                wabs[i] = mk[i] ? fabsf(wv[i]) : 0.0f;
+            }
+            acc[2 * kExpUnits] += (wabs[0] + wabs[1]) + (wabs[2] + wabs[3]);
+            acc[2 * kExpUnits + 1] += (float)((int)mk[0] + (int)mk[1] + (int)mk[2] + (int)mk[3]);
+#pragma unroll
+            for (int j = 0; j < kExpUnits; ++j) {
+                float s1 = 0.0f, s2 = 0.0f;
+                if (j < nu) {
+                    const float t[4] = {__uint_as_float(av[p][j].x), __uint_as_float(av[p][j].y), __uint_as_float(av[p][j].z),
+                                        __uint_as_float(av[p][j].w)};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        s1 += mk[i] ? t[i] : 0.0f;
+                        s2 = fmaf(wabs[i], mk[i] ? t[i] : 0.0f, s2);
+                    }
+                }
+                acc[2 * j] += s1;
+                acc[2 * j + 1] += s2;
+            }
+        }
+    }
+    for (int st = 0; !(VEC && !FUSED) && st < a.steps; ++st) {
         const int64_t piece = (int64_t)tile * a.steps + st;
         if (piece * kExpTile >= a.n_tok)
             break;
@@ -734,10 +816,39 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
         const int j = tid >> 1, which = tid & 1;
         if (j < kExpUnits) {
             if (j < nu) a.part[((int64_t)(u0 + j) * a.ntiles + tile) * 2 + which] = t;
+        } else if (a.done != nullptr) { // single-launch form: every unit group keeps its own copy of the token sums
+            a.part[((int64_t)(a.U + blockIdx.y) * a.ntiles + tile) * 2 + which] = t;
         } else if (blockIdx.y == 0) {
             a.part[((int64_t)a.U * a.ntiles + tile) * 2 + which] = t;
         }
     }
+    if (a.done == nullptr)
+        return;
+    // Single-launch form.  Every CTA publishes its partials and counts itself on its unit group's counter; the one
+    // that counts last has all partials of the group in view: its eight warps add those of the group's eight units
+    // in the order of exposure_final_kernel (so the results do not depend on which CTA that is) and take the units'
+    // plan decisions.  It leaves the counter at zero.
+    __shared__ bool s_last;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0)
+        s_last = atomicAdd(a.done + blockIdx.y, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last)
+        return;
+    __threadfence();
+    if (wid < nu) {
+        const int u = u0 + wid;
+        double s3;
+        const float E = exposure_of_unit(a.part, a.U + blockIdx.y, a.ntiles, u, a.eps_alpha, lane, &s3);
+        if (lane == 0) {
+            a.exposure[u] = E;
+            if (u == 0 && a.sum_abs_omega) *a.sum_abs_omega = (float)s3;
+            if (a.plan.avail) decide_unit(a.plan, u, &E);
+        }
+    }
+    if (tid == 0)
+        a.done[blockIdx.y] = 0;
 }
 
 // One warp per unit adds the per-tile partials in a fixed order and applies the closed form
@@ -746,22 +857,12 @@ __global__ void __launch_bounds__(32) exposure_final_kernel(const double *part, 
                                                             float *exposure, float *sum_abs_omega)
 {
     const int u = blockIdx.x, lane = threadIdx.x;
-    double s1 = 0.0, s2 = 0.0, s3 = 0.0, cnt = 0.0;
-    for (int t = lane; t < ntiles; t += 32) {
-        s1 += part[((int64_t)u * ntiles + t) * 2];
-        s2 += part[((int64_t)u * ntiles + t) * 2 + 1];
-        s3 += part[((int64_t)U * ntiles + t) * 2];
-        cnt += part[((int64_t)U * ntiles + t) * 2 + 1];
-    }
-    s1 = warp_sum(s1);
-    s2 = warp_sum(s2);
-    s3 = warp_sum(s3);
-    cnt = warp_sum(cnt);
+    grid_dependency_wait();
+    grid_dependency_release();
+    double s3;
+    const float E = exposure_of_unit(part, U, ntiles, u, eps_alpha, lane, &s3);
     if (lane == 0) {
-        double E = 0.0;
-        if (cnt > 0.0)
-            E = (s2 + (double)eps_alpha * s3) / (s1 / cnt + (double)eps_alpha);
-        exposure[u] = (float)E;
+        exposure[u] = E;
         if (u == 0 && sum_abs_omega) *sum_abs_omega = (float)s3;
     }
 }
@@ -913,12 +1014,22 @@ extern "C" size_t hilore_workspace_bytes(int32_t U, int64_t n_tok)
     return (size_t)(U + 1) * (size_t)(ntiles > 0 ? ntiles : 1) * 2 * sizeof(double);
 }
 
+// Single-launch form: partial sums of the U units and one row of token sums per unit group, then the counters.
+static size_t scores_plan_partial_bytes(int32_t U, int64_t n_tok)
+{
+    const int64_t ntiles = (n_tok + kExpTile - 1) / kExpTile;
+    const size_t groups = ((size_t)U + kExpUnits - 1) / kExpUnits;
+    return ((size_t)U + groups) * (size_t)(ntiles > 0 ? ntiles : 1) * 2 * sizeof(double);
+}
+extern "C" size_t hilore_scores_plan_workspace_bytes(int32_t U, int64_t n_tok);
+
 // fused: compute omega inside the reduction (hilore_coeffs_exposure); *fused_done tells the caller whether that was
 // possible for this shape (otherwise nothing has been launched and the caller runs the two passes in turn).
 static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T, int64_t n_tok,
                            const int32_t *cu, int64_t n_seq, const float *row_rms, int32_t U, int64_t rms_ld,
                            int32_t row_shift, float eps_alpha, float *exposure, float *sum_abs_omega, void *workspace,
-                           size_t workspace_bytes, void *stream, const FusedCoeff *fused = nullptr, bool *fused_done = nullptr)
+                           size_t workspace_bytes, void *stream, const FusedCoeff *fused = nullptr, bool *fused_done = nullptr,
+                           const PlanTail *plan = nullptr, bool single_launch = false)
 {
     if (n_rows < 0 || T < 0 || n_tok < 0 || U < 0 || row_shift < 0 || row_shift > 1)
         return HILORE_INVALID_ARG;
@@ -933,7 +1044,8 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     if (!aligned(workspace, 16) || !aligned(omega, 4) || !aligned(row_rms, 4) || !aligned(exposure, 4) ||
         !aligned(sum_abs_omega, 4) || !aligned(cu, 4))
         return HILORE_ALIGN;
-    if (workspace_bytes < hilore_workspace_bytes(U, n_tok))
+    const size_t part_bytes = single_launch ? scores_plan_partial_bytes(U, n_tok) : hilore_workspace_bytes(U, n_tok);
+    if (workspace_bytes < (single_launch ? hilore_scores_plan_workspace_bytes(U, n_tok) : part_bytes))
         return HILORE_WORKSPACE;
     const int64_t pieces = (n_tok + kExpTile - 1) / kExpTile;
     const int64_t groups = (U + kExpUnits - 1) / kExpUnits;
@@ -968,21 +1080,35 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     a.cu = cu;
     a.n_seq = (int)n_seq;
     a.steps = steps;
+    a.eps_alpha = eps_alpha;
+    a.exposure = exposure;
+    a.sum_abs_omega = sum_abs_omega;
+    if (single_launch && a.ntiles > 0) { // the counter of finished CTAs sits behind the partials and starts at zero
+        a.done = reinterpret_cast<unsigned int *>(static_cast<unsigned char *>(workspace) + part_bytes);
+        if (plan) a.plan = *plan;
+        if (cudaMemsetAsync(a.done, 0, sizeof(unsigned int) * (size_t)groups, st) != cudaSuccess)
+            return HILORE_CUDA;
+    }
     if (a.ntiles > 0) {
         const dim3 grid((unsigned)a.ntiles, (unsigned)((U + kExpUnits - 1) / kExpUnits));
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
                          aligned(mask, 4) && aligned(row_rms, 16);
+        void (*kernel)(ExpArgs) = nullptr;
         if (fused) {
             const bool fvec = vec && aligned(fused->logp_new, 16) && aligned(fused->logp_old, 16) && aligned(fused->logp_ref, 16) &&
                               aligned(fused->omega_out, 16);
-            if (fvec) exposure_partial_kernel<true, true><<<grid, kExpThreads, 0, st>>>(a);
-            else exposure_partial_kernel<false, true><<<grid, kExpThreads, 0, st>>>(a);
-        } else if (vec) exposure_partial_kernel<true><<<grid, kExpThreads, 0, st>>>(a);
-        else exposure_partial_kernel<false><<<grid, kExpThreads, 0, st>>>(a);
-        if (cudaGetLastError() != cudaSuccess)
+            kernel = fvec ? exposure_partial_kernel<true, true> : exposure_partial_kernel<false, true>;
+        } else {
+            kernel = vec ? exposure_partial_kernel<true, false> : exposure_partial_kernel<false, false>;
+        }
+        if (launch_dependent(kernel, grid, dim3(kExpThreads), 0, st, a) != cudaSuccess || cudaGetLastError() != cudaSuccess)
             return HILORE_CUDA;
     }
-    exposure_final_kernel<<<(unsigned)U, 32, 0, st>>>(a.part, U, a.ntiles, eps_alpha, exposure, sum_abs_omega);
+    if (a.done != nullptr) // the partial kernel's last CTA has finished the reduction (and the plan)
+        return HILORE_OK;
+    if (launch_dependent(exposure_final_kernel, dim3((unsigned)U), dim3(32), 0, st, (const double *)a.part, (int)U, a.ntiles, eps_alpha,
+                         exposure, sum_abs_omega) != cudaSuccess)
+        return HILORE_CUDA;
     return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
 }
 
@@ -1046,6 +1172,79 @@ extern "C" int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total
         return st;
     return launch_exposure(omega, mask, n_rows, T, n_tok, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha, exposure,
                            sum_abs_omega, workspace, workspace_bytes, stream);
+}
+
+extern "C" size_t hilore_scores_plan_workspace_bytes(int32_t U, int64_t n_tok)
+{
+    if (U < 0 || n_tok < 0)
+        return 0;
+    const size_t groups = ((size_t)U + kExpUnits - 1) / kExpUnits;
+    return scores_plan_partial_bytes(U, n_tok) + ((groups * sizeof(unsigned int) + 15) & ~(size_t)15);
+}
+
+extern "C" int hilore_scores_plan(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset, int64_t n_rows,
+                                  int64_t T, const float *logp_new, const float *logp_old, const float *logp_ref,
+                                  const uint8_t *mask, int64_t N_norm, const int64_t *N_norm_dev, float clip_eps, float beta,
+                                  float adv_eps, const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift,
+                                  float eps_alpha, float *omega, float *exposure, float *sum_abs_omega,
+                                  const hilore_unit *units_dev, const float *kappa, const float *ebar, float tau_lo, float tau_hi,
+                                  const uint8_t *avail, uint8_t *action_io, float *psi, uint8_t *recompute,
+                                  uint64_t *retained_bytes, void *workspace, size_t workspace_bytes, void *stream)
+{
+    // the argument rules of the calls it stands for
+    if (rewards == nullptr || n_resp_total < 0 || G <= 0 || resp_offset < 0 || n_rows < 0 || T < 0 || U <= 0)
+        return HILORE_INVALID_ARG;
+    if (n_resp_total % G != 0 || resp_offset + n_rows > n_resp_total || T % 4 != 0)
+        return HILORE_SHAPE;
+    if (beta != 0.0f && logp_ref == nullptr)
+        return HILORE_INVALID_ARG;
+    if (N_norm_dev == nullptr && N_norm <= 0)
+        return HILORE_ZERO_NORM;
+    const int64_t n_tok = n_rows * T;
+    if (n_tok <= 0 || logp_new == nullptr || logp_old == nullptr || mask == nullptr || omega == nullptr)
+        return HILORE_INVALID_ARG;
+    if (units_dev == nullptr || kappa == nullptr || ebar == nullptr || avail == nullptr || action_io == nullptr)
+        return HILORE_INVALID_ARG;
+    if (!aligned(logp_new, 16) || !aligned(logp_old, 16) || !aligned(logp_ref, 16) || !aligned(omega, 16) || !aligned(mask, 4) ||
+        !aligned(rewards, 4) || !aligned(N_norm_dev, 8) || !aligned(units_dev, 8) || !aligned(kappa, 4) || !aligned(ebar, 4) ||
+        !aligned(psi, 4) || !aligned(retained_bytes, 8))
+        return HILORE_ALIGN;
+    FusedCoeff f{};
+    f.rewards = rewards;
+    f.G = G;
+    f.resp_offset = resp_offset;
+    f.logp_new = logp_new;
+    f.logp_old = logp_old;
+    f.logp_ref = beta != 0.0f ? logp_ref : nullptr;
+    f.N_norm = N_norm;
+    f.N_norm_dev = reinterpret_cast<const long long *>(N_norm_dev);
+    f.clip_eps = clip_eps;
+    f.beta = beta;
+    f.adv_eps = adv_eps;
+    f.omega_out = omega;
+    PlanTail plan{};
+    plan.units = units_dev;
+    plan.kappa = kappa;
+    plan.ebar = ebar;
+    plan.tau_lo = tau_lo;
+    plan.tau_hi = tau_hi;
+    plan.avail = avail;
+    plan.action_io = action_io;
+    plan.psi = psi;
+    plan.recompute = recompute;
+    plan.retained_bytes = retained_bytes;
+    bool fused_done = false;
+    int st = launch_exposure(omega, mask, n_rows, T, n_tok, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha, exposure,
+                             sum_abs_omega, workspace, workspace_bytes, stream, &f, &fused_done, &plan, true);
+    if (st != HILORE_OK || fused_done)
+        return st;
+    // shapes the one-sweep kernel does not take: the coefficient pass, then the reduction and the plan in one launch
+    st = launch_coeffs(rewards, n_resp_total, G, resp_offset, n_rows, T, logp_new, logp_old, logp_ref, mask, N_norm, N_norm_dev,
+                       clip_eps, beta, adv_eps, 0, nullptr, omega, nullptr, nullptr, stream);
+    if (st != HILORE_OK)
+        return st;
+    return launch_exposure(omega, mask, n_rows, T, n_tok, nullptr, 0, row_rms, U, rms_ld, row_shift, eps_alpha, exposure,
+                           sum_abs_omega, workspace, workspace_bytes, stream, nullptr, nullptr, &plan, true);
 }
 
 extern "C" int hilore_unit_exposure_packed(const float *omega, const uint8_t *mask, int64_t n_tok,

@@ -22,7 +22,7 @@ def test_bench_line_has_the_contract_keys():
                 "vs_baseline", "dtype", "data", "config", "gpu_launches", "clocks", "roofline", "e2e"):
         assert key in d, key
     assert d["steps"] == 4 and d["warmup"] == 3 and d["n_gpus"] == 1 and d["vs_baseline"] is None
-    assert d["gpu_launches"] == 6 * 4 and "workload" in d["config"] and "model" not in d["config"]
+    assert d["gpu_launches"] == 4 * 4 and "workload" in d["config"] and "model" not in d["config"]
     assert d["config"]["workload"].startswith("7B-shaped") and d["config"]["plan_matches_thresholds"] is True
     assert d["sustained"]["seconds"] >= 0.3 and d["sustained"]["clocks"]["samples"] >= 3
     r = d["roofline"]
