@@ -55,6 +55,9 @@ __device__ __forceinline__ void prefetch_l2_bulk(const void *p, uint32_t bytes)
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 
+// Ask for the cache line that holds *p to be brought into L2; nothing waits for it.
+__device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 // Programmatic dependent launch: block until the kernels this one depends on have completed and their writes are
 // visible (a no-op when the kernel was launched without the attribute); and tell the next kernel of the stream that
 // it may start to become resident.
