@@ -170,7 +170,7 @@ size_t hilore_scores_plan_workspace_bytes(int32_t U, int64_t n_tok);
  *   adv_out      [n_seq] fp32, REQUIRED here: the per-sequence advantages are written by a first launch and read
  *                by the token kernel (2 launches).
  *   Exposure: the activation row of token k is k - row_shift; with row_shift = 1 a token whose source row
- *   would fall before the start of its own sequence has no activation term (it still counts in |T_b|).
+ *   would fall before the start of its own sequence carries no weight (it counts neither in the mean nor in E_u).
  *   Other arguments, status codes and workspace as in the dense calls.
  */
 int hilore_grpo_coeffs_packed(const float *rewards, int64_t n_resp_total, int32_t G, int64_t resp_offset,
@@ -223,7 +223,9 @@ size_t hilore_omega_diagnostics_workspace_bytes(void);
  *     E_u = sum_{t in T_b} |omega_t| alpha_{t,u};       |T_b| = 0  =>  E_u = 0
  * a_{t,u} is row_rms[u*rms_ld + i*T + t - row_shift] for slot (i, t): row_shift = 1 takes the
  * activation row of the source position that predicts token t (the paper's wording), 0 the
- * token's own row.  Slots with t - row_shift < 0 are skipped.
+ * token's own row.  A slot with t - row_shift < 0 has no activation row in this grid and carries no
+ * weight: it counts neither in abar_u nor in E_u (the weights of the other slots of T_b average to
+ * one); sum_abs_omega still covers all of T_b.
  *
  *   omega, mask   [n_rows, T] fp32 / u8 of the microbatch.    row_rms  [U, rms_ld] fp32, rms_ld >= n_rows*T.
  *   exposure      [U] fp32.     sum_abs_omega  opt, one fp32: sum_{t in T_b} |omega_t|.

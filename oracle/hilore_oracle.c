@@ -258,7 +258,9 @@ int orc_row_rms(const uint16_t *x, int64_t rows, int64_t cols, int64_t ld, float
 /* ------------------------------------------------------ a4: update exposure */
 /* alpha_t = (a_t + eps) / (mean_{s in T_b} a_s + eps);  E_u = sum_{t in T_b} |omega_t| alpha_t
  * (Eqs. "activation-token-weights", "mlp-weighted-exposure").  T_b = slots with mask = 1.
- * The activation row of slot (i, t) is (i, t - row_shift).  |T_b| = 0 => E_u = 0.         */
+ * The activation row of slot (i, t) is (i, t - row_shift); a slot whose row would lie before the start of
+ * its response carries no weight: it counts neither in the mean nor in E_u (so the weights of the slots
+ * that do have a row average to one, as Eq. "activation-token-weights" requires).  No such slot => E_u = 0. */
 int orc_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T, const float *row_rms,
                       int32_t U, int64_t rms_ld, int32_t row_shift, float eps_alpha, float *exposure,
                       float *sum_abs_omega)
@@ -269,13 +271,15 @@ int orc_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, i
         return ORC_INVALID;
     if (rms_ld < n_rows * T)
         return ORC_SHAPE;
-    int64_t cnt = 0;
+    int64_t cnt = 0; /* tokens of T_b that have an activation row: the weights average to one over these */
     double sw = 0.0;
-    for (int64_t k = 0; k < n_rows * T; ++k)
-        if (mask[k]) {
-            ++cnt;
-            sw += fabs((double)omega[k]);
-        }
+    for (int64_t i = 0; i < n_rows; ++i)
+        for (int64_t t = 0; t < T; ++t)
+            if (mask[i * T + t]) {
+                if (t - row_shift >= 0)
+                    ++cnt;
+                sw += fabs((double)omega[i * T + t]);
+            }
     if (sum_abs_omega)
         *sum_abs_omega = (float)sw;
     for (int32_t u = 0; u < U; ++u) {
@@ -658,7 +662,7 @@ int orc_grpo_coeffs_packed(const float *adv, const int32_t *cu_seqlens, int64_t 
 }
 
 /* orc_unit_exposure on the packed layout: the activation row of token k is k - row_shift, taken only when it
- * lies inside the token's own sequence. */
+ * lies inside the token's own sequence; a token without such a row carries no weight (see orc_unit_exposure). */
 int orc_unit_exposure_packed(const float *omega, const uint8_t *mask, const int32_t *cu_seqlens, int64_t n_seq,
                              const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift, float eps_alpha,
                              float *exposure, float *sum_abs_omega)
@@ -670,13 +674,15 @@ int orc_unit_exposure_packed(const float *omega, const uint8_t *mask, const int3
     const int64_t n_tok = cu_seqlens[n_seq];
     if (rms_ld < n_tok)
         return ORC_SHAPE;
-    int64_t cnt = 0;
+    int64_t cnt = 0; /* tokens of T_b whose activation row lies inside their own sequence */
     double sw = 0.0;
-    for (int64_t k = 0; k < n_tok; ++k)
-        if (mask[k]) {
-            ++cnt;
-            sw += fabs((double)omega[k]);
-        }
+    for (int64_t i = 0; i < n_seq; ++i)
+        for (int64_t k = cu_seqlens[i]; k < cu_seqlens[i + 1]; ++k)
+            if (mask[k]) {
+                if (k - row_shift >= cu_seqlens[i])
+                    ++cnt;
+                sw += fabs((double)omega[k]);
+            }
     if (sum_abs_omega)
         *sum_abs_omega = (float)sw;
     for (int32_t u = 0; u < U; ++u) {

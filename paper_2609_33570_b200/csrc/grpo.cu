@@ -823,7 +823,8 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
             }
         }
         acc[2 * kExpUnits] += (wabs[0] + wabs[1]) + (wabs[2] + wabs[3]);
-        acc[2 * kExpUnits + 1] += (float)((int)mk[0] + (int)mk[1] + (int)mk[2] + (int)mk[3]);
+        // the weights average to one over the slots of T_b that have an activation row: those are counted
+        acc[2 * kExpUnits + 1] += (float)((int)has[0] + (int)has[1] + (int)has[2] + (int)has[3]);
 #pragma unroll
         for (int j = 0; j < kExpUnits; ++j) {
             float s1 = 0.0f, s2 = 0.0f;

@@ -301,3 +301,29 @@ def test_coefficients_at_the_top_of_the_sweep_on_sampled_responses():
                             ro.mask[rows], ro.lengths[rows])
         check_coeffs(sub, got, N=ro.n_valid, beta=beta)
         assert not bool((omega == 7.0).any()) and not bool((a_out == 7.0).any())      # every slot and response written
+
+
+def test_exposure_shifted_rows_with_a_valid_first_slot():
+    """row_shift = 1 and the first slot of every response in T_b: the slot has no activation row and carries no weight
+    (neither in the mean nor in the sum); dense and packed layouts against the oracle."""
+    ro = synth.rollout(81, 3, 4, 96, rewards="uniform", lengths="uniform", min_len=5)
+    assert ro.mask[:, 0].all()
+    rng = np.random.default_rng(82)
+    omega = (rng.standard_normal((ro.n_resp, ro.T)) * 1e-4).astype(np.float32) * ro.mask
+    rms = rng.random((5, ro.n_resp * ro.T), dtype=np.float32) + np.float32(0.25)
+    E, sw = G.unit_exposure(omega, ro.mask, rms, row_shift=1)
+    oE, osw = oracle.unit_exposure(omega, ro.mask, rms, row_shift=1)
+    assert G.rel_err(E, oE).max() <= RTOL and abs(sw - osw) <= RTOL * osw
+    const = np.where(ro.mask != 0, np.float32(2e-4), 0).astype(np.float32)       # mean-one weights over the slots with a row
+    Ec, _ = G.unit_exposure(const, ro.mask, rms, row_shift=1, eps_alpha=0.0)
+    assert G.rel_err(Ec, np.full(5, 2e-4 * int(ro.mask[:, 1:].sum()))).max() <= RTOL
+    # packed: every sequence starts with its first response token (no prompt), so the same slots lack a row
+    pk = synth.pack_rollout(ro, 83, max_prompt=0, min_prompt=0)
+    om_p = np.concatenate([omega[i, :ro.lengths[i]] for i in range(ro.n_resp)]).astype(np.float32)
+    rms_p = rng.random((5, pk.n_tok), dtype=np.float32) + np.float32(0.25)
+    nws = api.hilore_workspace_bytes(5, pk.n_tok)
+    ws, Eg = G.Guarded(nws), G.Guarded(5 * 4)
+    api.hilore_unit_exposure_packed(G.dev(om_p), G.dev(pk.mask), pk.n_tok, G.dev(pk.cu_seqlens), len(pk.rows), G.dev(rms_p), 5,
+                                    pk.n_tok, 1, 1e-8, Eg.ptr(), None, ws.ptr(), nws)
+    oEp, _ = oracle.unit_exposure_packed(om_p, pk.mask, pk.cu_seqlens, rms_p, row_shift=1)
+    assert G.rel_err(Eg.numpy(np.float32, (5,)), oEp).max() <= RTOL

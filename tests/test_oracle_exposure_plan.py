@@ -99,6 +99,27 @@ def test_exposure_row_shift_uses_previous_position():
     np.testing.assert_allclose(E_shift, E_ref, rtol=1e-7)
 
 
+def test_exposure_row_shift_weights_average_to_one_over_the_slots_that_have_a_row():
+    """row_shift = 1 with the first slot of every response valid: that slot has no source row inside the grid and
+    carries no weight; over the remaining slots of T_b the weights average to one (Eq. activation-token-weights), so
+    constant |omega| = c gives E = c * (number of valid slots with t >= 1), whatever the activation magnitudes; and
+    the result equals the exposure of the same record with the first column masked out."""
+    omega, mask, rms = _case(7)
+    mask[:, 0] = 1
+    n_rows, T = omega.shape
+    c = np.float32(3e-4)
+    const = np.where(mask != 0, c, 0).astype(np.float32)
+    E, sw = oracle.unit_exposure(const, mask, rms, row_shift=1, eps_alpha=0.0)
+    with_row = int(mask[:, 1:].sum())
+    np.testing.assert_allclose(E, np.float64(c) * with_row, rtol=1e-6)
+    assert sw == pytest.approx(float(c) * int(mask.sum()), rel=1e-6)          # sum |omega| is over all of T_b
+    mask2 = mask.copy()
+    mask2[:, 0] = 0
+    E_a, _ = oracle.unit_exposure(omega * (mask != 0), mask, rms, row_shift=1)
+    E_b, _ = oracle.unit_exposure(omega * (mask2 != 0), mask2, rms, row_shift=1)
+    np.testing.assert_allclose(E_a, E_b, rtol=1e-6)
+
+
 def _avail_table():
     """Eq. "available-recovery-actions": q = H -> {H, L, R}; q = L -> {L, R}; q = R -> {R}."""
     return {ACT_H: {ACT_H, ACT_L, ACT_R}, ACT_L: {ACT_L, ACT_R}, ACT_R: {ACT_R}}

@@ -72,12 +72,13 @@ def test_exposure_hand_worked_first_token_rule():
     rms = np.array([[1, 2, 3, 4]], f32)
     E0, sw = oracle.unit_exposure_packed(omega, mask, cu, rms, row_shift=0, eps_alpha=0.0)
     assert E0[0] == pytest.approx(4.0, rel=1e-7) and sw == 4.0          # mean-one weights: E = sum |omega|
-    # row_shift = 1: tokens 0 and 2 have no source row inside their sequence; tokens 1, 3 read rows 0, 2
-    E1, _ = oracle.unit_exposure_packed(omega, mask, cu, rms, row_shift=1, eps_alpha=0.0)
-    assert E1[0] == pytest.approx((1 + 3) / ((1 + 3) / 4), rel=1e-7)
-    # one long sequence: only token 0 is skipped
+    # row_shift = 1: tokens 0 and 2 have no source row inside their sequence and carry no weight; tokens 1, 3 read
+    # rows 0, 2 (a = 1, 3): mean 2, E = (1 * 1 + 1 * 3) / 2 -- the two weights 1/2 and 3/2 average to one
+    E1, sw1 = oracle.unit_exposure_packed(omega, mask, cu, rms, row_shift=1, eps_alpha=0.0)
+    assert E1[0] == pytest.approx((1 + 3) / ((1 + 3) / 2), rel=1e-7) and sw1 == 4.0
+    # one long sequence: only token 0 is skipped; a = 1, 2, 3 with mean 2
     E2, _ = oracle.unit_exposure_packed(omega, mask, np.array([0, 4], np.int32), rms, row_shift=1, eps_alpha=0.0)
-    assert E2[0] == pytest.approx((1 + 2 + 3) / ((1 + 2 + 3) / 4), rel=1e-7)
+    assert E2[0] == pytest.approx((1 + 2 + 3) / ((1 + 2 + 3) / 3), rel=1e-7)
 
 
 @pytest.mark.parametrize("row_shift", [0, 1])
