@@ -38,10 +38,15 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     if (FMT < 0 || FMT == HILORE_FMT_INT8_BLK) fill_scale_table<HILORE_FMT_INT8_BLK>(sm_tab[1]);
     grid_dependency_wait();    // everything above touched shared memory only
     grid_dependency_release(); // the next kernel's CTAs may take the place of ours as they finish
-    __syncthreads();           // scale tables are filled
+    // descriptors and gates of the launch once into shared memory: a CTA that meets a new unit every few iterations
+    // would otherwise wait for a dependent global load before it can issue the unit's first data loads (+5 % on
+    // the 1.5B-shaped table, +7 % on the token-RMS capture of the 7B-shaped one)
+    __shared__ UnitStage stage;
+    stage_units(wk, false, stage);
+    __syncthreads();           // scale tables and descriptors are in place
     JobCursor cur;
     Job j;
-    while (next_job(wk, nullptr, false, cur, j, kBlockSumSlots)) {
+    while (next_job(wk, &stage, false, cur, j, kBlockSumSlots)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
         if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[0]);
         else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[0]);

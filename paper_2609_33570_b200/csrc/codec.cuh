@@ -151,8 +151,7 @@ struct JobCursor {
     bool tail_done = false;
 };
 
-// `st`: the staged descriptors (recover kernel), or nullptr: descriptors and gates are read from global memory at
-// every unit (compress kernel: its register budget is full, and the staged form cost more in the hot loop).
+// `st`: the staged descriptors, or nullptr: descriptors and gates are read from global memory at every unit.
 __device__ __forceinline__ bool next_job(const CodecWork &wk, const UnitStage *st, bool recover, JobCursor &cur, Job &j, int slots)
 {
     const uint32_t nC = gridDim.x;
