@@ -46,7 +46,7 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     __syncthreads();           // scale tables and descriptors are in place
     JobCursor cur;
     Job j;
-    while (next_job(wk, &stage, false, cur, j, kBlockSumSlots)) {
+    while (next_job(wk, stage, cur, j, kBlockSumSlots)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
         if (fmt == HILORE_FMT_E4M3FN_RAW) compress_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[0]);
         else if (fmt == HILORE_FMT_E4M3FN_BLK) compress_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.op, j.r0, j.r1, j.rows_per_batch, sm_blocksum, sm_tab[0]);
@@ -75,7 +75,7 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_k
     uint32_t tile = 0;
     JobCursor cur;
     Job j;
-    while (next_job(wk, &stage, true, cur, j, 0)) {
+    while (next_job(wk, stage, cur, j, 1)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
         if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
         else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);

@@ -68,38 +68,6 @@ constexpr int kStageUnits = 96;
 constexpr int kIterChunks = 2 * kCodecThreads;       // chunks one iteration of a CTA covers (16 KB of bf16)
 constexpr int kFlatCols = kIterChunks * 16;          // a 16 KB piece seen as one row of 8192 elements
 
-struct UnitStage {
-    hilore_unit u[kStageUnits];
-    int op[kStageUnits];
-};
-
-// Stage the launch's units: what to do with each (OP_NONE if the launch is not gated into it or it lacks a
-// buffer the operation needs) and its descriptor.  `recover`: which of the two kernels is asking.
-__device__ __forceinline__ void stage_units(const CodecWork &wk, bool recover, UnitStage &st)
-{
-    for (int t = threadIdx.x; t < wk.U; t += blockDim.x) {
-        int op = unit_op(wk, t);
-        if (recover ? (op != OP_RECOVER) : (op != OP_COMPRESS && op != OP_STATS))
-            op = OP_NONE;
-        if (op != OP_NONE) {
-            hilore_unit u = wk.units ? wk.units[t] : wk.single;
-            const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
-            if ((op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (op == OP_STATS && (!u.x || !u.row_rms)) ||
-                (op == OP_RECOVER && (!u.out || !u.codes || (scaled && !u.scales))))
-                op = OP_NONE; // the unit lacks a buffer this operation needs: leave it untouched
-            if (op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
-                u.row_rms = nullptr; // token magnitudes were collected at capture time
-            st.u[t] = u;
-        }
-        st.op[t] = op;
-    }
-}
-
-__device__ __forceinline__ uint64_t share_multiplier(const CodecWork &wk, uint32_t c) // floor(c * 2^32 / nC), c <= nC
-{
-    return (uint64_t)c * wk.share_m + (c * wk.share_rem) / gridDim.x;
-}
-
 struct UnitPlan {
     int64_t items;     // rows or 16 KB pieces
     int64_t seg_items; // items per window
@@ -135,6 +103,40 @@ __device__ __forceinline__ UnitPlan plan_unit(const CodecWork &wk, const hilore_
     return p;
 }
 
+struct UnitStage {
+    hilore_unit u[kStageUnits];
+    int op[kStageUnits];
+    UnitPlan plan[kStageUnits]; // how each unit is shared among the CTAs (worked out once per kernel, not per CTA visit)
+};
+
+// Stage the launch's units: what to do with each (OP_NONE if the launch is not gated into it or it lacks a
+// buffer the operation needs), its descriptor and its sharing plan.  `recover`: which of the two kernels is asking.
+__device__ __forceinline__ void stage_units(const CodecWork &wk, bool recover, UnitStage &st)
+{
+    for (int t = threadIdx.x; t < wk.U; t += blockDim.x) {
+        int op = unit_op(wk, t);
+        if (recover ? (op != OP_RECOVER) : (op != OP_COMPRESS && op != OP_STATS))
+            op = OP_NONE;
+        if (op != OP_NONE) {
+            hilore_unit u = wk.units ? wk.units[t] : wk.single;
+            const bool scaled = u.fmt != HILORE_FMT_E4M3FN_RAW;
+            if ((op == OP_COMPRESS && (!u.x || !u.codes || (scaled && !u.scales))) || (op == OP_STATS && (!u.x || !u.row_rms)) ||
+                (op == OP_RECOVER && (!u.out || !u.codes || (scaled && !u.scales))))
+                op = OP_NONE; // the unit lacks a buffer this operation needs: leave it untouched
+            if (op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
+                u.row_rms = nullptr; // token magnitudes were collected at capture time
+            st.u[t] = u;
+            st.plan[t] = plan_unit(wk, u, !recover && u.row_rms != nullptr);
+        }
+        st.op[t] = op;
+    }
+}
+
+__device__ __forceinline__ uint64_t share_multiplier(const CodecWork &wk, uint32_t c) // floor(c * 2^32 / nC), c <= nC
+{
+    return (uint64_t)c * wk.share_m + (c * wk.share_rem) / gridDim.x;
+}
+
 // One piece of work of a CTA: rows [r0, r1) of a unit (or of the 16 KB-piece view of it), in batches of
 // `rows_per_batch` rows where per-row sums are collected.
 struct Job {
@@ -151,30 +153,16 @@ struct JobCursor {
     bool tail_done = false;
 };
 
-// `st`: the staged descriptors, or nullptr: descriptors and gates are read from global memory at every unit.
-__device__ __forceinline__ bool next_job(const CodecWork &wk, const UnitStage *st, bool recover, JobCursor &cur, Job &j, int slots)
+// The next piece of work of this CTA, from the staged descriptors, gates and sharing plans of the launch.
+__device__ __forceinline__ bool next_job(const CodecWork &wk, const UnitStage &st, JobCursor &cur, Job &j, int slots)
 {
     const uint32_t nC = gridDim.x;
     for (; cur.ui < wk.U; ++cur.ui, cur.seg_item = 0, cur.tail_done = false) {
-        if (st) {
-            j.op = st->op[cur.ui];
-            if (j.op == OP_NONE)
-                continue;
-            j.u = st->u[cur.ui];
-        } else {
-            j.op = unit_op(wk, cur.ui);
-            if (recover ? (j.op != OP_RECOVER) : (j.op != OP_COMPRESS && j.op != OP_STATS))
-                continue;
-            j.u = wk.units ? wk.units[cur.ui] : wk.single;
-            const bool scaled = j.u.fmt != HILORE_FMT_E4M3FN_RAW;
-            if ((j.op == OP_COMPRESS && (!j.u.x || !j.u.codes || (scaled && !j.u.scales))) ||
-                (j.op == OP_STATS && (!j.u.x || !j.u.row_rms)) || (j.op == OP_RECOVER && (!j.u.out || !j.u.codes || (scaled && !j.u.scales))))
-                continue; // the unit lacks a buffer this operation needs: leave it untouched
-            if (j.op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
-                j.u.row_rms = nullptr; // token magnitudes were collected at capture time
-        }
-        const bool per_row = !recover && j.u.row_rms != nullptr;
-        const UnitPlan p = plan_unit(wk, j.u, per_row);
+        j.op = st.op[cur.ui];
+        if (j.op == OP_NONE)
+            continue;
+        j.u = st.u[cur.ui];
+        const UnitPlan p = st.plan[cur.ui];
         const int nb = (int)(j.u.cols >> 6);
         while (cur.seg_item < p.items) {
             const int64_t s0 = cur.seg_item, n = min(p.seg_items, p.items - s0);
