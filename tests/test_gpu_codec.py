@@ -139,6 +139,29 @@ def test_stats_only_and_no_stats():
     assert none is None and np.array_equal(codes, o_codes) and np.array_equal(scales, o_scales)
 
 
+@pytest.mark.parametrize("fmt", FMTS)
+def test_codes_only_pass_on_16KB_pieces_with_special_values_and_a_ragged_tail(fmt):
+    """Without the token RMS a contiguous unit is shared as 16 KB pieces (rows do not matter) plus one short tail:
+    77 x 1536 elements = 14 pieces and 144 chunks.  Special values sit in whole pieces and in the tail."""
+    rng = np.random.default_rng(17)
+    x = synth.activation_unit(rng, 77, 1536)
+    x[0, 5] = 0x7FC0                                   # NaN in the first piece
+    x[3, 70] = 0x7F80                                  # +Inf
+    x[40, 640:704] = 0                                 # an all-zero block
+    x[41, 0] = 0x43E9                                  # 466: overflows to NaN in the unscaled cast
+    x[76, 1500] = 0xFF80                               # -Inf in the tail
+    x[76, 1535] = 0xFFC0                               # NaN in the last element
+    codes, scales, none = G.compress(x, fmt, want_rms=False)
+    o_codes, o_scales = oracle.compress(x, fmt, 0 if fmt == api.FMT_E4M3FN_RAW else 64)
+    assert none is None and np.array_equal(codes, o_codes)
+    if o_scales is not None:
+        assert np.array_equal(scales.view(np.uint32), o_scales.view(np.uint32))
+    got = G.recover(codes, scales, fmt)
+    want = oracle.recover(o_codes, o_scales, fmt, 0 if fmt == api.FMT_E4M3FN_RAW else 64)
+    nan = lambda b: (b & 0x7FFF) > 0x7F80
+    assert np.array_equal(nan(got), nan(want)) and np.array_equal(got[~nan(want)], want[~nan(want)])
+
+
 def test_run_to_run_determinism():
     x = synth.activation_unit(np.random.default_rng(8), 4096, 3584)
     a = G.compress(x, api.FMT_E4M3FN_BLK)
