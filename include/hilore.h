@@ -96,7 +96,9 @@ int hilore_mask_count(const uint8_t *mask, int64_t n, int64_t *count, void *stre
  *   resp_offset, n_rows   this call covers responses [resp_offset, resp_offset + n_rows), a microbatch
  *                of the rollout batch; a prompt group may straddle two calls.
  *   logp_new, logp_old, logp_ref   [n_rows, T] fp32, 16-byte aligned; logp_ref may be NULL iff beta == 0.
- *   mask         [n_rows, T] u8 (0 / 1), 4-byte aligned.  T % 4 must be 0 (HILORE_SHAPE).
+ *   mask         [n_rows, T] u8 (0 / 1), 4-byte aligned.  T % 4 must be 0 (HILORE_SHAPE).  With T % 8 == 0, the fp32
+ *                tensors 32-byte aligned and the byte tensors 8-byte aligned the call takes its fast path (256-bit
+ *                accesses, one warp per 512 slots); the results do not depend on the path.
  *   N_norm, N_norm_dev   the normaliser N: if N_norm_dev (one int64 on the device, e.g. written by
  *                hilore_mask_count earlier on the same stream) is not NULL it is read by the kernel and
  *                N_norm is ignored; a device value <= 0 yields omega = 0 everywhere.  Otherwise N_norm
@@ -135,7 +137,7 @@ int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G
  * that finishes last among those of a group of eight units adds the group's per-tile partial sums in the fixed order
  * of the two-kernel form and takes the plan decisions of its units, so omega, exposure, psi, action_io, recompute and retained_bytes are bit for bit those of
  * the separate calls, whichever CTA that is.  Between forward and backward of a microbatch this is one launch (plus a
- * 4-byte memset) instead of four.
+ * memset of one counter per unit group) instead of four.
  *   Arguments as in hilore_coeffs_exposure (omega REQUIRED, U > 0, n_rows * T > 0) and in the DECIDE phase of
  *   hilore_plan_apply (units_dev, kappa, ebar, avail, action_io REQUIRED; psi, recompute, retained_bytes opt; the
  *   unit table is only read for rows, cols and fmt, on the device).

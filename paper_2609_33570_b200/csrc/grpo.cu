@@ -64,36 +64,11 @@ constexpr int kCoeffTile = kCoeffThreads * kCoeffVec * 4;     // 1024 slots of o
 // d_0 = 0 the subtraction loses at most a factor G of the 2^-53 relative precision; and all rewards are the same
 // number exactly when S2 == 0, which is the test for an equal-reward group.
 struct GroupStats {
-    double r0, mu, inv_den; // mu: mean of the shifted rewards; inv_den = 1 / (sigma + adv_eps)
+    double r0, mu, sigma; // mu is the mean of the shifted rewards
     bool equal;
 };
 
-// 1 / d and 1 / sqrt(v) in fp64 from an fp32 seed and two Newton steps (relative error below 1e-15): a handful of
-// FMAs instead of the 40-60 instructions of an IEEE fp64 division or square root.  Every warp of the coefficient
-// kernels evaluates the statistics of its own tile, so this sequence is a third of their instructions otherwise.
-// Valid while the operand is a normal fp32 number; the callers fall back to the IEEE operations outside that range.
-__device__ __forceinline__ bool in_fp32_range(double x) { return x > 1e-36 && x < 1e36; }
-__device__ __forceinline__ double recip64(double d)
-{
-    if (!in_fp32_range(d))
-        return 1.0 / d;
-    double y = (double)__frcp_rn((float)d);
-    y = fma(y, fma(-d, y, 1.0), y);
-    y = fma(y, fma(-d, y, 1.0), y);
-    return y;
-}
-__device__ __forceinline__ double sqrt64(double v)
-{
-    if (!in_fp32_range(v))
-        return sqrt(v);
-    double y = (double)rsqrtf((float)v);
-    const double h = 0.5 * v;
-    y = fma(y, fma(-h * y, y, 0.5), y);
-    y = fma(y, fma(-h * y, y, 0.5), y);
-    return v * y;
-}
-
-__device__ __forceinline__ GroupStats group_stats(const float *R, int G, float adv_eps, int lane)
+__device__ __forceinline__ GroupStats group_stats(const float *R, int G, int lane)
 {
     GroupStats g;
     g.r0 = (double)__ldg(R);
@@ -107,27 +82,25 @@ __device__ __forceinline__ GroupStats group_stats(const float *R, int G, float a
     s2 = warp_sum(s2);
     g.equal = s2 == 0.0;
     g.mu = 0.0;
-    g.inv_den = 0.0;
+    g.sigma = 0.0;
     if (g.equal)
         return g;
-    const double inv_G = recip64((double)G);
-    g.mu = s1 * inv_G;
-    const double sigma = sqrt64(fmax((s2 - s1 * g.mu) * inv_G, 0.0));
-    g.inv_den = recip64(sigma + (double)adv_eps);
+    g.mu = s1 / (double)G;
+    g.sigma = sqrt(fmax((s2 - s1 * g.mu) / (double)G, 0.0));
     return g;
 }
 
 // Advantage of a response with reward `r`: exactly zero in an equal-reward group, whatever the rounding of the mean.
-__device__ __forceinline__ float advantage_of(const GroupStats &g, float r)
+__device__ __forceinline__ float advantage_of(const GroupStats &g, float r, float adv_eps)
 {
-    return g.equal ? 0.0f : (float)((((double)r - g.r0) - g.mu) * g.inv_den);
+    return g.equal ? 0.0f : (float)((((double)r - g.r0) - g.mu) / (g.sigma + (double)adv_eps));
 }
 
 // Advantage of response `resp`, from the G rewards of its prompt group (one warp).
 __device__ __forceinline__ float group_advantage(const float *rewards, int64_t resp, int G, float adv_eps, int lane)
 {
-    const GroupStats g = group_stats(rewards + (resp / G) * G, G, adv_eps, lane);
-    return advantage_of(g, __ldg(rewards + resp));
+    const GroupStats g = group_stats(rewards + (resp / G) * G, G, lane);
+    return advantage_of(g, __ldg(rewards + resp), adv_eps);
 }
 
 constexpr float kLog2e = 1.4426950408889634f;
@@ -221,7 +194,7 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_kernel(const __grid
         const float A = group_advantage(a.rewards, a.resp_offset + row, a.G, a.adv_eps, lane);
         if (lane == 0) {
             const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
-            const double invN = N > 0 ? recip64((double)N) : 0.0;
+            const double invN = N > 0 ? 1.0 / (double)N : 0.0;
             s_adv = A;
             s_coef = (float)(-(double)A * invN); // omega = coef * r on the unclipped branch
             s_nkl = -(float)((double)a.beta * invN);
@@ -378,7 +351,7 @@ __global__ void __launch_bounds__(kCoeffThreads, KL ? HILORE_COEFF_MINB_KL : HIL
     grid_dependency_release();
     const float A = group_advantage(a.rewards, a.resp_offset + row, a.G, a.adv_eps, lane);
     const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
-    const double invN = N > 0 ? recip64((double)N) : 0.0;
+    const double invN = N > 0 ? 1.0 / (double)N : 0.0;
     const float coef = (float)(-(double)A * invN);
     const float nkl = -(float)((double)a.beta * invN);
     if (tt == 0 && lane == 0 && a.adv_out)
@@ -439,11 +412,11 @@ __global__ void __launch_bounds__(128) packed_advantage_kernel(const float *rewa
     const int lane = threadIdx.x & 31;
     const int64_t g = resp_offset / G + (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
     if (g * G >= resp_offset + n_seq) return;
-    const GroupStats st = group_stats(rewards + g * G, G, adv_eps, lane);
+    const GroupStats st = group_stats(rewards + g * G, G, lane);
     for (int j = lane; j < G; j += 32) {
         const int64_t resp = g * G + j;
         if (resp >= resp_offset && resp < resp_offset + n_seq)
-            adv[resp - resp_offset] = advantage_of(st, __ldg(rewards + resp));
+            adv[resp - resp_offset] = advantage_of(st, __ldg(rewards + resp), adv_eps);
     }
 }
 
@@ -501,7 +474,7 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_packed_kernel(const
     __shared__ double s_invN;
     if (tid == 64) { // the fp64 reciprocal of the normaliser once per CTA
         const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
-        s_invN = N > 0 ? recip64((double)N) : 0.0;
+        s_invN = N > 0 ? 1.0 / (double)N : 0.0;
     }
     if (tid < 64) {
         const int64_t first = (int64_t)blockIdx.x * kCoeffTile;
@@ -683,7 +656,7 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
         row_lo = slot_lo / a.T;
         const int nrows = (int)((slot_hi - 1) / a.T - row_lo) + 1;
         const long long N = a.f.N_norm_dev ? *a.f.N_norm_dev : (long long)a.f.N_norm;
-        const double invN = N > 0 ? recip64((double)N) : 0.0;
+        const double invN = N > 0 ? 1.0 / (double)N : 0.0;
         for (int r = wid; r < nrows; r += kExpThreads / 32) {
             const float A = group_advantage(a.f.rewards, a.f.resp_offset + row_lo + r, a.f.G, a.f.adv_eps, lane);
             if (lane == 0) {

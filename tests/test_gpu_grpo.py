@@ -327,3 +327,28 @@ def test_exposure_shifted_rows_with_a_valid_first_slot():
                                     pk.n_tok, 1, 1e-8, Eg.ptr(), None, ws.ptr(), nws)
     oEp, _ = oracle.unit_exposure_packed(om_p, pk.mask, pk.cu_seqlens, rms_p, row_shift=1)
     assert G.rel_err(Eg.numpy(np.float32, (5,)), oEp).max() <= RTOL
+
+
+@pytest.mark.parametrize("beta", [0.0, 0.02])
+def test_fast_and_generic_coefficient_paths_give_the_same_bits(beta):
+    """T % 8 == 0 and 32-byte alignment select the warp-per-tile kernel (256-bit accesses, packed fp32 pairs), anything
+    else the 128-bit one: the same inputs at 32-byte and at 16-byte aligned addresses must give identical omega, ratio
+    and clip indicator, masked slots included."""
+    ro = synth.rollout(91, 6, 8, 1096, rewards="uniform", lengths="uniform", min_len=3)
+    ro.logp_ref[:] = ro.logp_new + np.random.default_rng(92).normal(0, 0.2, ro.logp_new.shape).astype(np.float32)
+    n, T = ro.n_resp, ro.T
+
+    def run(shift):                                   # shift in elements: 0 -> 32-byte aligned, 4 -> only 16-byte
+        pad = lambda a, dt: torch.cat([torch.zeros(shift, dtype=dt, device="cuda"), torch.from_numpy(a.reshape(-1)).cuda()])[shift:]
+        big = lambda dt: torch.zeros(n * T + 8, dtype=dt, device="cuda")[shift:shift + n * T]
+        ln, lo, lr = (pad(a, torch.float32) for a in (ro.logp_new, ro.logp_old, ro.logp_ref))
+        mk = torch.cat([torch.zeros(2 * shift, dtype=torch.uint8, device="cuda"), torch.from_numpy(ro.mask.reshape(-1)).cuda()])[2 * shift:]
+        omega, ratio, chi = big(torch.float32), big(torch.float32), torch.zeros(n * T + 16, dtype=torch.uint8, device="cuda")[2 * shift:2 * shift + n * T]
+        assert ln.data_ptr() % 32 == (16 if shift else 0)
+        api.hilore_grpo_coeffs(G.dev(ro.rewards), n, ro.G, 0, n, T, ln, lo, lr if beta else None, mk, ro.n_valid, None, 0.2, beta,
+                               1e-6, None, omega, ratio, chi)
+        return omega.cpu().numpy(), ratio.cpu().numpy(), chi.cpu().numpy()
+
+    fast, generic = run(0), run(4)
+    for a, b in zip(fast, generic):
+        assert a.tobytes() == b.tobytes()
