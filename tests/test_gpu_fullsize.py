@@ -78,6 +78,54 @@ def test_bench_step_1p5B_shaped_microbatch():
     torch.cuda.empty_cache()
 
 
+def test_bench_step_7B_shaped_mixed_plan():
+    """configs[2], the exact object bench.py times as its headline: 84 units [16384, 3584|3584|18944], capture with
+    the candidate plan all H, `hilore_scores_plan` with the microbatch's thresholds (42 L / 25 H / 17 R), encode and
+    recovery of the L units.  Every expected value comes from the oracle's own chain on the host inputs."""
+    dev = torch.device("cuda", 0)
+    cfg = bench.CONFIGS[3]
+    wl = bench.Workload(api, synth, cfg, seed=0, device=dev)
+    wl.prepare_plan()
+    for t in wl.codes:
+        t.fill_(0xA5)
+    for t in wl.scales:
+        t.fill_(-7.0)
+    for t in wl.out:
+        t.fill_(-3.0)
+    mb = 5
+    wl.step(mb)
+    torch.cuda.synchronize()
+    a = wl.action.cpu().numpy()
+    assert np.array_equal(a, wl.expected_action[mb]) and [(a == v).sum() for v in (L, H, R)] == [42, 25, 17]
+    assert np.array_equal(wl.recompute.cpu().numpy(), (a == R).astype(np.uint8))
+    ro = wl.ro
+    sl = slice(mb * cfg["mb_resp"], (mb + 1) * cfg["mb_resp"])
+    adv = oracle.group_advantages(ro.rewards, ro.G)
+    w, _, _ = oracle.grpo_coeffs(adv[sl], ro.logp_new[sl], ro.logp_old[sl], None, ro.mask[sl], N_norm=ro.n_valid)
+    assert G.rel_err(wl.omega.cpu().numpy(), w).max() <= 1e-5
+    sample = [0, 1, 41, 82, 5]                             # four narrow units and one wide one
+    o_rms = np.stack([oracle.row_rms(bits(wl.x[u])) for u in sample])
+    assert G.rel_err(wl.rms.cpu().numpy()[sample], o_rms).max() <= 1e-5
+    oE, _ = oracle.unit_exposure(w, ro.mask[sl], o_rms)
+    assert G.rel_err(wl.exposure.cpu().numpy()[sample], oE).max() <= 1e-5
+    kappa, ebar = wl.kappa.cpu().numpy()[sample], wl.ebar.cpu().numpy()[sample]
+    oa, opsi, orec, oret = oracle.plan(oE, kappa, ebar, wl.tau[mb][0], wl.tau[mb][1], [H] * len(sample),
+                                       [wl.shapes[u][0] for u in sample], [wl.shapes[u][1] for u in sample], [1] * len(sample),
+                                       [64] * len(sample))
+    assert G.rel_err(wl.psi.cpu().numpy()[sample], opsi).max() <= 1e-5
+    assert np.array_equal(a[sample], oa) and np.array_equal(wl.retained.cpu().numpy()[sample].view(np.uint64), oret)
+    rng = np.random.default_rng(9)
+    narrow_L = [u for u in range(wl.U) if a[u] == L and wl.shapes[u][1] < 10000]
+    wide_L = [u for u in range(wl.U) if a[u] == L and wl.shapes[u][1] > 10000]
+    for u in narrow_L[:2] + narrow_L[-1:] + wide_L[:1] + wide_L[-1:]:
+        check_rows(wl.x[u], wl.codes[u], wl.scales[u], wl.out[u], wl.rms[u], sample_rows(rng, wl.rows, 8), api.FMT_E4M3FN_BLK)
+    for u in [v for v in range(wl.U) if a[v] != L][:10]:      # H keeps its bundle, R is recomputed: nothing written
+        assert bool((wl.codes[u][::257] == 0xA5).all()) and bool((wl.scales[u][::257] == -7.0).all())
+        assert bool((wl.out[u][::257] == -3.0).all())
+    del wl
+    torch.cuda.empty_cache()
+
+
 def test_7B_shaped_mixed_plan():
     """configs[2]: 84 units [16384, 3584|3584|18944], candidate plan all H, thresholds at the 50 % / 70 %
     quantiles of psi (42 L / 17 R / 25 H), post-forward encode and recovery of the L units only."""
