@@ -12,7 +12,10 @@ pytestmark = pytest.mark.gpu
 L, H, R = api.ACT_L, api.ACT_H, api.ACT_R
 
 
-def test_step_captured_in_a_cuda_graph_and_replayed_on_new_data():
+@pytest.mark.parametrize("one_launch", [False, True])
+def test_step_captured_in_a_cuda_graph_and_replayed_on_new_data(one_launch):
+    """one_launch: the score refresh through hilore_scores_plan (a kernel and the memset of its counters) instead of
+    the coefficient, exposure and decide calls."""
     dev = torch.device("cuda", 0)
     rng = np.random.default_rng(0)
     shapes = [(256, 896), (256, 1536), (256, 4864)]
@@ -35,16 +38,21 @@ def test_step_captured_in_a_cuda_graph_and_replayed_on_new_data():
     action = torch.zeros(U, dtype=torch.uint8, device=dev)
     kappa = torch.ones(U, dtype=torch.float32, device=dev)
     ebar = torch.full((U,), 0.025, dtype=torch.float32, device=dev)
-    nws = api.hilore_workspace_bytes(U, rows)
+    nws = api.hilore_scores_plan_workspace_bytes(U, rows)
     ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
 
     def step(stream):
         api.hilore_plan_apply(udev, uhost, U, api.PHASE_CAPTURE, None, None, None, 0, 0, avail, action, None, None, None, stream=stream)
-        api.hilore_grpo_coeffs(rewards, 4, 4, 0, 4, 64, lp, lo, None, mask, ro.n_valid, None, 0.2, 0.0, 1e-6, None, omega, None,
-                               None, stream=stream)
-        api.hilore_unit_exposure(omega, mask, 4, 64, rms, U, rows, 0, 1e-8, expo, None, ws, nws, stream=stream)
-        api.hilore_plan_apply(udev, uhost, U, api.PHASE_DECIDE, expo, kappa, ebar, float("inf"), float("inf"), avail, action, psi,
-                              None, None, stream=stream)
+        if one_launch:
+            api.hilore_scores_plan(rewards, 4, 4, 0, 4, 64, lp, lo, None, mask, ro.n_valid, None, 0.2, 0.0, 1e-6, rms, U, rows, 0,
+                                   1e-8, omega, expo, None, udev, kappa, ebar, float("inf"), float("inf"), avail, action, psi,
+                                   None, None, ws, nws, stream=stream)
+        else:
+            api.hilore_grpo_coeffs(rewards, 4, 4, 0, 4, 64, lp, lo, None, mask, ro.n_valid, None, 0.2, 0.0, 1e-6, None, omega,
+                                   None, None, stream=stream)
+            api.hilore_unit_exposure(omega, mask, 4, 64, rms, U, rows, 0, 1e-8, expo, None, ws, nws, stream=stream)
+            api.hilore_plan_apply(udev, uhost, U, api.PHASE_DECIDE, expo, kappa, ebar, float("inf"), float("inf"), avail, action,
+                                  psi, None, None, stream=stream)
         api.hilore_plan_apply(udev, uhost, U, api.PHASE_ENCODE, None, None, None, 0, 0, avail, action, None, None, None, stream=stream)
         api.hilore_plan_apply(udev, uhost, U, api.PHASE_RECOVER, None, None, None, 0, 0, avail, action, None, None, None, stream=stream)
 
