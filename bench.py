@@ -242,14 +242,14 @@ class Workload:
             self.bytes_encode = [0] * self.n_plan
             self.bytes_recover = [0] * self.n_plan
             self.expected_action = [None] * self.n_plan
-            self.launches_per_step = 4   # capture, scores + plan, encode, recover (and one 4-byte memset)
+            self.launches_per_step = 4   # capture, scores + plan, encode, recover
         else:
             self.bytes_capture = sum(codec_bytes(r, c, True, True) for r, c in self.shapes)
             self.n_plan = self.n_microbatches
             self.tau = [(inf, inf)] * self.n_plan
             self.bytes_encode = [0] * self.n_plan
             self.bytes_recover = [sum(codec_bytes(r, c, True, False) for r, c in self.shapes)] * self.n_plan
-            self.launches_per_step = 3   # capture, scores + plan, recover (and one 4-byte memset)
+            self.launches_per_step = 3   # capture, scores + plan, recover
 
     def bytes_step(self, mb):
         mb %= self.n_plan

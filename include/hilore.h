@@ -133,16 +133,18 @@ int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G
 /*
  * The score refresh of one microbatch in ONE kernel launch: hilore_coeffs_exposure followed by
  * hilore_plan_apply(HILORE_PHASE_DECIDE) (Algorithm 1, lines "coefficients", "exposure", risk score and allocation;
- * Eqs. "update-coefficient", "mlp-weighted-exposure", "token-weighted-risk", "available-recovery-actions").  The CTA
- * that finishes last among those of a group of eight units adds the group's per-tile partial sums in the fixed order
- * of the two-kernel form and takes the plan decisions of its units, so omega, exposure, psi, action_io, recompute and retained_bytes are bit for bit those of
- * the separate calls, whichever CTA that is.  Between forward and backward of a microbatch this is one launch (plus a
- * memset of one counter per unit group) instead of four.
+ * Eqs. "update-coefficient", "mlp-weighted-exposure", "token-weighted-risk", "available-recovery-actions").  The CTAs of
+ * a group of eight units -- one per tile of 1024 tokens -- add their partial sums in the fixed order of the two-kernel
+ * form and one of them takes the plan decisions of the group's units, so omega, exposure, psi, action_io, recompute and
+ * retained_bytes are bit for bit those of the separate calls.  At microbatch size (1, 2, 4, 8 or 16 tiles) the CTAs of a
+ * group are one thread-block cluster and exchange the sums through its distributed shared memory; otherwise through
+ * the workspace, the CTA that finishes last (a counter per group, cleared by a memset inside the call) doing the
+ * rest.  Between forward and backward of a microbatch this is one launch instead of four.
  *   Arguments as in hilore_coeffs_exposure (omega REQUIRED, U > 0, n_rows * T > 0) and in the DECIDE phase of
  *   hilore_plan_apply (units_dev, kappa, ebar, avail, action_io REQUIRED; psi, recompute, retained_bytes opt; the
  *   unit table is only read for rows, cols and fmt, on the device).
  *   workspace   at least hilore_scores_plan_workspace_bytes(U, n_rows * T) bytes, 16-byte aligned: the partial sums
- *               and, behind them, the counters of finished CTAs, which the call sets to zero itself.
+ *               and, behind them, the counters of finished CTAs (unused by the cluster form).
  *   Microbatches beyond the one-sweep form's limits (see hilore_coeffs_exposure) run the coefficient pass first and
  *   then the reduction + plan launch.
  */

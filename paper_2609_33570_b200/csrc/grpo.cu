@@ -3,6 +3,8 @@
 // the proof of Prop. 1, Eq. "activation-token-weights" and Eq. "mlp-weighted-exposure".
 #include "common.cuh"
 
+#include <cooperative_groups.h>
+
 namespace hilore {
 
 // ------------------------------------------------------------------ N = sum of the update mask
@@ -551,6 +553,20 @@ constexpr int kExpUnits = 8;              // units per CTA (omega and mask are r
 // One warp adds the per-tile partials of unit u in a fixed order and applies the closed form
 //   E_u = (S2_u + eps * S3) / (S1_u / |T_b| + eps),  S1 = sum a, S2 = sum |omega| a, S3 = sum |omega|.
 // Every lane returns E_u; *s3_out gets S3.
+// The closed form from the per-lane sums over the tiles (lane t holds the sums of tiles t, t + 32, ...).
+__device__ __forceinline__ float exposure_from_lane_sums(double s1, double s2, double s3, double cnt, float eps_alpha, double *s3_out)
+{
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    s3 = warp_sum(s3);
+    cnt = warp_sum(cnt);
+    double E = 0.0;
+    if (cnt > 0.0)
+        E = (s2 + (double)eps_alpha * s3) / (s1 / cnt + (double)eps_alpha);
+    *s3_out = s3;
+    return (float)E;
+}
+
 __device__ __forceinline__ float exposure_of_unit(const double *part, int tok_row, int ntiles, int u, float eps_alpha, int lane,
                                                   double *s3_out)
 {
@@ -561,15 +577,7 @@ __device__ __forceinline__ float exposure_of_unit(const double *part, int tok_ro
         s3 += __ldcg(part + ((int64_t)tok_row * ntiles + t) * 2);
         cnt += __ldcg(part + ((int64_t)tok_row * ntiles + t) * 2 + 1);
     }
-    s1 = warp_sum(s1);
-    s2 = warp_sum(s2);
-    s3 = warp_sum(s3);
-    cnt = warp_sum(cnt);
-    double E = 0.0;
-    if (cnt > 0.0)
-        E = (s2 + (double)eps_alpha * s3) / (s1 / cnt + (double)eps_alpha);
-    *s3_out = s3;
-    return (float)E;
+    return exposure_from_lane_sums(s1, s2, s3, cnt, eps_alpha, s3_out);
 }
 
 // Inputs of the coefficient pass when it is fused into the exposure reduction (hilore_coeffs_exposure).
@@ -601,6 +609,7 @@ struct ExpArgs {
     FusedCoeff f;      // used by the fused kernel only
     // single-launch form: the CTA that finishes last adds the partials and, if asked, takes the plan decisions
     unsigned int *done; // counter of finished CTAs (zero before the launch), or nullptr: a second kernel finishes
+    int cluster;        // 1: the CTAs of a unit group form one thread-block cluster and reduce through its shared memory
     float eps_alpha;
     float *exposure, *sum_abs_omega;
     PlanTail plan;      // plan.avail == nullptr: no decisions
@@ -830,17 +839,51 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
         if (lane == 0) sm[wid][q] = (double)v;
     }
     __syncthreads();
+    __shared__ double s_part[2 * (kExpUnits + 1)]; // this CTA's partial sums, for the cluster form
     if (tid < 2 * (kExpUnits + 1)) {
         double t = 0.0;
         for (int w = 0; w < kExpThreads / 32; ++w) t += sm[w][tid];
         const int j = tid >> 1, which = tid & 1;
-        if (j < kExpUnits) {
+        s_part[tid] = t;
+        if (a.cluster) {
+            // the sums stay in shared memory
+        } else if (j < kExpUnits) {
             if (j < nu) a.part[((int64_t)(u0 + j) * a.ntiles + tile) * 2 + which] = t;
         } else if (a.done != nullptr) { // single-launch form: every unit group keeps its own copy of the token sums
             a.part[((int64_t)(a.U + blockIdx.y) * a.ntiles + tile) * 2 + which] = t;
         } else if (blockIdx.y == 0) {
             a.part[((int64_t)a.U * a.ntiles + tile) * 2 + which] = t;
         }
+    }
+    if (a.cluster) {
+        // Cluster form of the single launch (microbatch sizes): the CTAs of a unit group -- one per tile of tokens --
+        // are one thread-block cluster.  After the cluster barrier the first CTA reads every CTA's partial sums from
+        // its shared memory (distributed shared memory), lane t taking tile t as the final kernel does, so the
+        // results are those of the other forms bit for bit; no partial sum goes through global memory, nothing is
+        // counted, nothing needs clearing.  A second barrier keeps the other CTAs' shared memory alive until then.
+        namespace cg = cooperative_groups;
+        cg::cluster_group cl = cg::this_cluster();
+        cl.sync();
+        if (cl.block_rank() == 0 && wid < nu) {
+            double s1 = 0.0, s2 = 0.0, s3 = 0.0, cnt = 0.0;
+            if (lane < (int)gridDim.x) {
+                const double *remote = cl.map_shared_rank(s_part, lane);
+                s1 = remote[2 * wid];
+                s2 = remote[2 * wid + 1];
+                s3 = remote[2 * kExpUnits];
+                cnt = remote[2 * kExpUnits + 1];
+            }
+            double s3_all;
+            const float E = exposure_from_lane_sums(s1, s2, s3, cnt, a.eps_alpha, &s3_all);
+            if (lane == 0) {
+                const int u = u0 + wid;
+                a.exposure[u] = E;
+                if (u == 0 && a.sum_abs_omega) *a.sum_abs_omega = (float)s3_all;
+                if (a.plan.avail) decide_unit(a.plan, u, &E);
+            }
+        }
+        cl.sync();
+        return;
     }
     if (a.done == nullptr)
         return;
@@ -1034,6 +1077,43 @@ extern "C" size_t hilore_workspace_bytes(int32_t U, int64_t n_tok)
     return (size_t)(U + 1) * (size_t)(ntiles > 0 ? ntiles : 1) * 2 * sizeof(double);
 }
 
+// Whether `kernel` may be launched with clusters of `size` CTAs on the current device (sizes above 8 need an opt-in
+// and enough SMs per GPC); asked once per kernel, size and device.
+template <typename K> static bool cluster_launch_ok(K kernel, int size)
+{
+    static std::mutex mu;
+    static struct { const void *k; int size, dev, ok; } seen[64];
+    static int n_seen = 0;
+    const int dev = current_device();
+    const void *key = reinterpret_cast<const void *>(kernel);
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < n_seen; ++i)
+        if (seen[i].k == key && seen[i].size == size && seen[i].dev == dev)
+            return seen[i].ok != 0;
+    int ok = 1;
+    if (size > 8 && cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+        ok = 0;
+    if (ok) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)size, 1);
+        cfg.blockDim = dim3(kExpThreads);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)size;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) != cudaSuccess || clusters < 1)
+            ok = 0;
+    }
+    (void)cudaGetLastError();
+    if (n_seen < 64)
+        seen[n_seen++] = {key, size, dev, ok};
+    return ok != 0;
+}
+
 // Single-launch form: partial sums of the U units and one row of token sums per unit group, then the counters.
 static size_t scores_plan_partial_bytes(int32_t U, int64_t n_tok)
 {
@@ -1103,6 +1183,42 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     a.eps_alpha = eps_alpha;
     a.exposure = exposure;
     a.sum_abs_omega = sum_abs_omega;
+    // Microbatch sizes: one thread-block cluster per unit group (up to 16 CTAs, one per tile), reduction through the
+    // cluster's shared memory; no counters, no memset.  Tile counts that are not a cluster size the device schedules
+    // (or a device that refuses the launch) take the counter form below.
+    if (single_launch && a.ntiles >= 1 && a.ntiles <= 16 && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
+        const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
+                         aligned(mask, 4) && aligned(row_rms, 16);
+        void (*kernel)(ExpArgs) = nullptr;
+        if (fused) {
+            const bool fvec = vec && aligned(fused->logp_new, 16) && aligned(fused->logp_old, 16) && aligned(fused->logp_ref, 16) &&
+                              aligned(fused->omega_out, 16);
+            kernel = fvec ? exposure_partial_kernel<true, true> : exposure_partial_kernel<false, true>;
+        } else {
+            kernel = vec ? exposure_partial_kernel<true, false> : exposure_partial_kernel<false, false>;
+        }
+        if (cluster_launch_ok(kernel, a.ntiles)) {
+            a.cluster = 1;
+            if (plan) a.plan = *plan;
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3((unsigned)a.ntiles, (unsigned)groups);
+            cfg.blockDim = dim3(kExpThreads);
+            cfg.stream = st;
+            cudaLaunchAttribute attr[2];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)a.ntiles;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[1].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 2;
+            if (cudaLaunchKernelEx(&cfg, kernel, a) == cudaSuccess && cudaGetLastError() == cudaSuccess)
+                return HILORE_OK;
+            (void)cudaGetLastError(); // refused: fall through to the counter form
+            a.cluster = 0;
+        }
+    }
     if (single_launch && a.ntiles > 0) { // the counter of finished CTAs sits behind the partials and starts at zero
         a.done = reinterpret_cast<unsigned int *>(static_cast<unsigned char *>(workspace) + part_bytes);
         if (plan) a.plan = *plan;
