@@ -54,6 +54,11 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) compress_
     }
 }
 
+// Tiles of bulk L2 prefetch run-ahead of the recover pass (8 KB of codes per tile and CTA).  Measured on B200 (TB/s
+// at run-ahead 0 / 1 / 2 / 3): block-scaled formats, whose decode waits for a scale as well, 4 GiB unit
+// 6.12 / 6.40 / 6.30, 7B-shaped table 5.98 / 6.36 / 6.32; the unscaled format, 4 GiB unit 6.21 / 6.08 / 6.02 / 6.02.
+constexpr int kPrefetchRecoverScaled = 1, kPrefetchRecoverUnscaled = 0;
+
 template <int FMT> __device__ __forceinline__ void recover_unit(const hilore_unit &u, int64_t r0, int64_t r1, uint8_t *sm_out,
                                                                 uint32_t &tile, int prefetch)
 {
@@ -77,9 +82,9 @@ template <int FMT> __global__ void __launch_bounds__(kCodecThreads, 4) recover_k
     Job j;
     while (next_job(wk, stage, cur, j, 1)) {
         const int fmt = FMT >= 0 ? FMT : j.u.fmt;
-        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
-        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
-        else recover_unit<HILORE_FMT_INT8_BLK>(j.u, j.r0, j.r1, sm_out, tile, wk.prefetch);
+        if (fmt == HILORE_FMT_E4M3FN_RAW) recover_unit<HILORE_FMT_E4M3FN_RAW>(j.u, j.r0, j.r1, sm_out, tile, kPrefetchRecoverUnscaled);
+        else if (fmt == HILORE_FMT_E4M3FN_BLK) recover_unit<HILORE_FMT_E4M3FN_BLK>(j.u, j.r0, j.r1, sm_out, tile, kPrefetchRecoverScaled);
+        else recover_unit<HILORE_FMT_INT8_BLK>(j.u, j.r0, j.r1, sm_out, tile, kPrefetchRecoverScaled);
     }
     if (threadIdx.x == 0)
         bulk_wait_all(); // every bulk store of this CTA is complete before it gives up its shared memory
@@ -126,17 +131,13 @@ static int check_unit(const hilore_unit &u, bool strict, bool need_x, bool need_
     return HILORE_OK;
 }
 
-// Tiles of bulk L2 prefetch run-ahead of the recover pass (8 KB of codes per tile and CTA): one to three measure
-// alike on B200, none is 6 % slower.
-constexpr int kPrefetchRecover = 2;
 // Window of a unit that all CTAs sweep together (see next_job).  Measured on B200: a 4 GiB unit runs at
 // 5.5 / 6.2 TB/s (compress / recover) uncut, 6.0 / 6.3 TB/s in windows of 64-96 MB; below about 48 MB the
 // pieces per CTA become too short.
 constexpr int64_t kSegmentBytes = 96ll << 20;
 
-template <typename K> static int launch_one(K kernel, CodecWork wk, int64_t total_rows, int prefetch, cudaStream_t st)
+template <typename K> static int launch_one(K kernel, CodecWork wk, int64_t total_rows, cudaStream_t st)
 {
-    wk.prefetch = prefetch;
     wk.seg_bytes = kSegmentBytes;
     int64_t grid = (int64_t)sm_count() * ctas_per_sm(kernel, kCodecThreads, 0, 2);
     if (grid > total_rows)
@@ -175,20 +176,18 @@ static int launch_codec(const CodecWork &wk, int64_t total_rows, int fmt, bool r
     if (total_rows <= 0)
         return HILORE_OK;
     if (recover) {
-        const int pf = kPrefetchRecover;
         switch (fmt) {
-        case HILORE_FMT_E4M3FN_RAW: return launch_one(recover_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, pf, st);
-        case HILORE_FMT_E4M3FN_BLK: return launch_one(recover_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, pf, st);
-        case HILORE_FMT_INT8_BLK: return launch_one(recover_kernel<HILORE_FMT_INT8_BLK>, wk, total_rows, pf, st);
-        default: return launch_one(recover_kernel<-1>, wk, total_rows, pf, st);
+        case HILORE_FMT_E4M3FN_RAW: return launch_one(recover_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, st);
+        case HILORE_FMT_E4M3FN_BLK: return launch_one(recover_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, st);
+        case HILORE_FMT_INT8_BLK: return launch_one(recover_kernel<HILORE_FMT_INT8_BLK>, wk, total_rows, st);
+        default: return launch_one(recover_kernel<-1>, wk, total_rows, st);
         }
     }
-    const int pf = 0; // the compress pass picks its run-ahead per unit (what it writes decides)
     switch (fmt) {
-    case HILORE_FMT_E4M3FN_RAW: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, pf, st);
-    case HILORE_FMT_E4M3FN_BLK: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, pf, st);
-    case HILORE_FMT_INT8_BLK: return launch_one(compress_kernel<HILORE_FMT_INT8_BLK>, wk, total_rows, pf, st);
-    default: return launch_one(compress_kernel<-1>, wk, total_rows, pf, st);
+    case HILORE_FMT_E4M3FN_RAW: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_RAW>, wk, total_rows, st);
+    case HILORE_FMT_E4M3FN_BLK: return launch_one(compress_kernel<HILORE_FMT_E4M3FN_BLK>, wk, total_rows, st);
+    case HILORE_FMT_INT8_BLK: return launch_one(compress_kernel<HILORE_FMT_INT8_BLK>, wk, total_rows, st);
+    default: return launch_one(compress_kernel<-1>, wk, total_rows, st);
     }
 }
 

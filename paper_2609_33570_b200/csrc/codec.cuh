@@ -26,7 +26,6 @@ struct CodecWork {
     int phase;                // HILORE_PHASE_* for table mode; CodecOp for single mode
     const uint8_t *avail;     // q_u
     const uint8_t *action;    // a_u
-    int prefetch;             // iterations of L2 prefetch run-ahead (0 = none)
     int64_t seg_bytes;        // size of the window all CTAs sweep together
     uint64_t share_m;         // 2^32 = share_m * grid + share_rem
     uint32_t share_rem;
