@@ -131,7 +131,8 @@ static int check_unit(const hilore_unit &u, bool strict, bool need_x, bool need_
     return HILORE_OK;
 }
 
-// Window of a unit that all CTAs sweep together (see next_job).  Measured on B200: a 4 GiB unit runs at
+// Scale of the windows of a unit that all CTAs sweep together (see plan_unit, next_job): units up to 1.5 x this size
+// go in one piece, larger ones in windows of two thirds of it or more.  Measured on B200: a 4 GiB unit runs at
 // 5.5 / 6.2 TB/s (compress / recover) uncut, 6.0 / 6.3 TB/s in windows of 64-96 MB; below about 48 MB the
 // pieces per CTA become too short.
 constexpr int64_t kSegmentBytes = 96ll << 20;
