@@ -297,6 +297,35 @@ def oracle_unit(xb: np.ndarray, threads=16):
     return tuple(np.concatenate([p[i] for p in parts]) for i in range(4))
 
 
+@pytest.mark.parametrize("rows,cols", [(16384, 18944), (36000, 4096), (20001, 8960)])
+def test_whole_units_that_are_shared_in_several_windows(rows, cols):
+    """Single units large enough to be cut into windows (rows of 37 KB, 8 KB and 17.5 KB; the last two with row counts
+    that leave uneven last windows), compared WHOLE with the oracle: compress with token RMS (row shares), compress
+    without it and recover (16 KB pieces).  A row or piece lost or done twice at a window or CTA boundary shows here."""
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(rows + cols)
+    x = synth.activation_unit_device(gen, rows, cols, dev)
+    oc, osc, oout, orms = oracle_unit(bits(x))
+    for with_rms in (True, False):
+        codes = torch.full((rows, cols), 0xA5, dtype=torch.uint8, device=dev)
+        scales = torch.full((rows, cols // 64), -7.0, dtype=torch.float32, device=dev)
+        rms = torch.full((rows,), -1.0, dtype=torch.float32, device=dev)
+        out = torch.full((rows, cols), -3.0, dtype=torch.bfloat16, device=dev)
+        api.hilore_compress(x, rows, cols, cols, api.FMT_E4M3FN_BLK, 64, codes, scales, rms if with_rms else None)
+        api.hilore_recover(codes, scales, rows, cols, api.FMT_E4M3FN_BLK, 64, out, cols)
+        torch.cuda.synchronize()
+        assert np.array_equal(codes.cpu().numpy(), oc)
+        assert np.array_equal(scales.cpu().numpy().view(np.uint32), osc.view(np.uint32))
+        assert np.array_equal(bits(out), oout)
+        if with_rms:
+            assert G.rel_err(rms.cpu().numpy(), orms).max() <= 1e-5
+        else:
+            assert bool((rms == -1.0).all())
+        del codes, scales, rms, out
+    torch.cuda.empty_cache()
+
+
 def test_1p5B_shaped_whole_units_and_checksums_over_microbatches():
     """configs[1]: the step bench.py's 1.5B-shaped leg times, on fresh activations per microbatch.  Microbatches 0 and
     63: one narrow and one wide unit compared WHOLE with the oracle (codes, scale bits, reconstruction, token RMS), and
