@@ -325,6 +325,62 @@ def exposure_case(log2_tok, U, reps):
     torch.cuda.synchronize()
 
 
+class ScoreRefresh:
+    """Inputs of one microbatch's score refresh (coefficients, exposure of U units, plan) at the 7B-shaped size: 16
+    responses of 1024 tokens, 84 units; only the token RMS of the units is needed, not the units themselves."""
+
+    def __init__(self, n_resp=16, T=1024, U=84, G=16):
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(9)
+        self.n_resp, self.T, self.U, self.G = n_resp, T, U, G
+        n_tok = n_resp * T
+        self.lp = torch.randn((n_resp, T), generator=gen, device="cuda") * 0.5 - 1.5
+        self.lo = self.lp + torch.randn((n_resp, T), generator=gen, device="cuda") * 0.05
+        self.mask = (torch.rand((n_resp, T), generator=gen, device="cuda") < 0.9).to(torch.uint8)
+        self.rewards = (torch.rand(n_resp, generator=gen, device="cuda") < 0.5).float()
+        self.rms = torch.rand((U, n_tok), generator=gen, device="cuda") + 0.5
+        self.omega = torch.empty((n_resp, T), device="cuda")
+        self.exposure, self.psi = torch.zeros(U, device="cuda"), torch.zeros(U, device="cuda")
+        self.kappa, self.ebar = torch.ones(U, device="cuda"), torch.full((U,), 0.03, device="cuda")
+        self.avail = torch.full((U,), api.ACT_H, dtype=torch.uint8, device="cuda")
+        self.action, self.recompute = torch.zeros(U, dtype=torch.uint8, device="cuda"), torch.zeros(U, dtype=torch.uint8, device="cuda")
+        self.retained = torch.zeros(U, dtype=torch.int64, device="cuda")
+        self.units_dev, self.units_host = api.make_unit_table(
+            [dict(rows=n_tok, cols=3584 if i % 3 else 18944, fmt=api.FMT_E4M3FN_BLK, block=64) for i in range(U)], "cuda")
+        self.ws_bytes = max(api.hilore_workspace_bytes(U, n_tok), api.hilore_scores_plan_workspace_bytes(U, n_tok))
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device="cuda")
+
+    def one_launch(self):
+        api.hilore_scores_plan(self.rewards, self.n_resp, self.G, 0, self.n_resp, self.T, self.lp, self.lo, None, self.mask,
+                               self.n_resp * self.T, None, 0.2, 0.0, 1e-6, self.rms, self.U, self.n_resp * self.T, 0, 1e-8,
+                               self.omega, self.exposure, None, self.units_dev, self.kappa, self.ebar, 1e-9, 1e-8, self.avail,
+                               self.action, self.psi, self.recompute, self.retained, self.ws, self.ws_bytes)
+
+    def separate_calls(self):
+        api.hilore_coeffs_exposure(self.rewards, self.n_resp, self.G, 0, self.n_resp, self.T, self.lp, self.lo, None, self.mask,
+                                   self.n_resp * self.T, None, 0.2, 0.0, 1e-6, self.rms, self.U, self.n_resp * self.T, 0, 1e-8,
+                                   self.omega, self.exposure, None, self.ws, self.ws_bytes)
+        api.hilore_plan_apply(self.units_dev, self.units_host, self.U, api.PHASE_DECIDE, self.exposure, self.kappa, self.ebar,
+                              1e-9, 1e-8, self.avail, self.action, self.psi, self.recompute, self.retained)
+
+
+def score_refresh_point(reps):
+    """The score refresh of a 7B-shaped microbatch (16384 tokens, 84 units): one launch against the separate calls."""
+    sr = ScoreRefresh()
+    a, b = time_calls([sr.one_launch], reps), time_calls([sr.separate_calls], reps)
+    return {"case": "score_refresh", "tokens": sr.n_resp * sr.T, "U": sr.U,
+            "one_launch_us": a["loop_ms"] * 1e3, "one_launch_device_us": a["device_us"], "one_launch_host_us": a["host_us"],
+            "separate_calls_us": b["loop_ms"] * 1e3, "separate_calls_device_us": b["device_us"],
+            "separate_calls_host_us": b["host_us"]}
+
+
+def score_refresh_case(reps):
+    sr = ScoreRefresh()
+    for _ in range(reps):
+        sr.one_launch()
+    torch.cuda.synchronize()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--cols", type=int, default=4096)
@@ -336,7 +392,7 @@ def main():
     ap.add_argument("--no-coeffs", action="store_true")
     ap.add_argument("--no-rms", action="store_true", help="compress without the fused token RMS")
     ap.add_argument("--plan-table", action="store_true", help="only the 7B-shaped table under several candidate plans")
-    ap.add_argument("--case", choices=["codec", "coeffs", "exposure"], help="run one small single-kernel case and exit")
+    ap.add_argument("--case", choices=["codec", "coeffs", "exposure", "scores"], help="run one small single-kernel case and exit")
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--fmt", type=int, default=api.FMT_E4M3FN_BLK)
     ap.add_argument("--units", type=int, default=2)
@@ -352,6 +408,8 @@ def main():
         coeffs_case(a.log2_slots, a.reps, a.beta)
     elif a.case == "exposure":
         exposure_case(a.log2_slots, a.U, a.reps)
+    elif a.case == "scores":
+        score_refresh_case(a.reps)
     if a.case:
         print("done")
         return
@@ -384,6 +442,7 @@ def main():
             print(json.dumps(diagnostics_point(ls, max(3, a.reps // 4))), flush=True)
         for U in (36, 84):
             print(json.dumps(allocate_point(U, max(3, a.reps // 4))), flush=True)
+        print(json.dumps(score_refresh_point(a.reps)), flush=True)
 
 
 if __name__ == "__main__":
