@@ -184,9 +184,10 @@ def coeffs_packed_point(log2_tokens, reps, G=8, mean_len=2048):
     omega = [torch.empty_like(x) for x in lp]
     fns = [lambda i=i: api.hilore_grpo_coeffs_packed(rewards, n_seq, G, 0, n_seq, cu, n_tok, lp[i], lo[i], None, mask, n_tok,
                                                      None, 0.2, 0.0, 1e-6, adv, omega[i], None, None) for i in range(pool)]
-    t = _time(fns, reps)
+    tc = time_calls(fns, reps)
+    t = tc["loop_ms"]
     return {"kernel": "grpo_coeffs_packed", "tokens": n_tok, "n_seq": n_seq, "pool": pool, "us": t * 1e3,
-            "tokens_per_s": n_tok / t * 1e3, "gbs": 13 * n_tok / t / 1e6}
+            "device_us": tc["device_us"], "host_us": tc["host_us"], "tokens_per_s": n_tok / t * 1e3, "gbs": 13 * n_tok / t / 1e6}
 
 
 def diagnostics_point(log2_slots, reps, G=16, T=1024):

@@ -170,9 +170,11 @@ size_t hilore_scores_plan_workspace_bytes(int32_t U, int64_t n_tok);
  *                cu_seqlens[n_seq] = n_tok.  The contents are the caller's responsibility (they are not read on
  *                the host); whatever they hold, no kernel indexes outside [0, n_seq] or [0, n_tok).
  *   logp_*, omega, ratio [n_tok] fp32, 16-byte aligned;  mask, clip_mask [n_tok] u8, 4-byte aligned; n_tok need
- *                not be a multiple of 4 (n_tok < 2^31).
+ *                not be a multiple of 4 (n_tok < 2^31).  With 32-byte aligned fp32 tensors and 8-byte aligned masks
+ *                the call takes its fast kernel (one warp per 512 tokens); the results are the same bits either way.
  *   adv_out      [n_seq] fp32, REQUIRED here: the per-sequence advantages are written by a first launch and read
- *                by the token kernel (2 launches).
+ *                by the token kernel (2 launches; the second starts while the first runs and waits for it only
+ *                before it uses an advantage).
  *   Exposure: the activation row of token k is k - row_shift; with row_shift = 1 a token whose source row
  *   would fall before the start of its own sequence carries no weight (it counts neither in the mean nor in E_u).
  *   Other arguments, status codes and workspace as in the dense calls.

@@ -413,6 +413,12 @@ __global__ void __launch_bounds__(128) packed_advantage_kernel(const float *rewa
 {
     const int lane = threadIdx.x & 31;
     const int64_t g = resp_offset / G + (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+    // Launched as a programmatic dependent: first everything ahead in the stream must be complete (a kernel of this
+    // library may still be reading the advantage array this kernel rewrites).  Then the coefficient kernel behind
+    // this one may start: it reads its token data and finds its sequences while this kernel runs, and waits for the
+    // advantages (griddepcontrol.wait) before it uses them.
+    grid_dependency_wait();
+    grid_dependency_release();
     if (g * G >= resp_offset + n_seq) return;
     const GroupStats st = group_stats(rewards + g * G, G, lane);
     for (int j = lane; j < G; j += 32) {
@@ -539,6 +545,126 @@ __global__ void __launch_bounds__(kCoeffThreads) grpo_coeffs_packed_kernel(const
                 if (EXTRA) {
                     if (a.ratio) a.ratio[k0[j] + i] = r[i];
                     if (a.clip_mask) a.clip_mask[k0[j] + i] = (uint8_t)((chi >> (8 * i)) & 1u);
+                }
+            }
+        }
+    }
+}
+
+// The packed fast path: one WARP per tile of kWarpTile tokens, as in the dense warp kernel (no CTA barrier, 256-bit
+// accesses, packed fp32 pairs).  The warp finds the owner of its first token with one cooperative search, then reads
+// the 32 sequence boundaries that follow it with one coalesced load: those that fall inside the tile tell every lane
+// its sequence by counting, without further loads (sequences of 1-3 K tokens: zero or one boundary per tile).  A lane
+// whose eight tokens lie in one sequence takes the packed arithmetic; one that straddles a boundary, or the ragged
+// end of the microbatch, walks its tokens one by one.  Same bits as the generic kernel.  Needs 32-byte aligned
+// tensors (8-byte masks).
+template <bool KL, bool EXTRA>
+__global__ void __launch_bounds__(kCoeffThreads, 6) grpo_coeffs_packed_warp_kernel(const __grid_constant__ PackedArgs a,
+                                                                                    uint32_t total_tiles)
+{
+    constexpr uint32_t kFull = 0xFFFFFFFFu;
+    const int lane = threadIdx.x & 31;
+    const uint32_t wt = blockIdx.x * (kCoeffThreads / 32) + (threadIdx.x >> 5);
+    if (wt >= total_tiles)
+        return;
+    const int64_t first = (int64_t)wt * kWarpTile;
+    // The kernel ahead in the stream computes the advantages and nothing else, and it lets this one start only after
+    // everything before it in the stream is complete: token data, masks, sequence boundaries and N are final already.
+    uint32_t sn[kWarpIters][8], so[kWarpIters][8], sr[KL ? kWarpIters : 1][8];
+    uint2 mk[kWarpIters];
+    int64_t k0[kWarpIters];
+    int cnt[kWarpIters];
+#pragma unroll
+    for (int i = 0; i < kWarpIters; ++i) {
+        k0[i] = first + i * 256 + lane * 8;
+        const int64_t left = a.n_tok - k0[i];
+        cnt[i] = left >= 8 ? 8 : (left > 0 ? (int)left : 0);
+        if (cnt[i] == 8) {
+            ld_global_256(a.logp_new + k0[i], sn[i]);
+            ld_global_256(a.logp_old + k0[i], so[i]);
+            if (KL) ld_global_256(a.logp_ref + k0[i], sr[i]);
+            mk[i] = ld_global_64_stream(a.mask + k0[i]);
+        } else { // ragged end of the microbatch: element by element, zeros beyond it
+            uint32_t m[2] = {0, 0};
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const bool in = e < cnt[i];
+                sn[i][e] = in ? __float_as_uint(a.logp_new[k0[i] + e]) : 0u;
+                so[i][e] = in ? __float_as_uint(a.logp_old[k0[i] + e]) : 0u;
+                if (KL) sr[i][e] = in ? __float_as_uint(a.logp_ref[k0[i] + e]) : 0u;
+                if (in && a.mask[k0[i] + e] != 0) m[e >> 2] |= 1u << (8 * (e & 3));
+            }
+            mk[i] = make_uint2(m[0], m[1]);
+        }
+    }
+    const int64_t last = min(first + kWarpTile, a.n_tok) - 1;
+    const int own = owner_sequence_warp(a.cu, a.n_seq, first, lane);
+    // lane j: the first token of sequence own + 1 + j (past the table: a value no token reaches)
+    const int bi = own + 1 + lane;
+    const int bound = bi <= a.n_seq ? __ldg(a.cu + bi) : 0x7FFFFFFF;
+    const int nle = __popc(__ballot_sync(kFull, (int64_t)bound <= last)); // sequences that begin inside the tile
+    const long long N = a.N_norm_dev ? *a.N_norm_dev : (long long)a.N_norm;
+    const double invN = N > 0 ? 1.0 / (double)N : 0.0;
+    const float nkl = -(float)((double)a.beta * invN);
+    const float hi = 1.0f + a.clip_eps, lo = 1.0f - a.clip_eps;
+    grid_dependency_wait(); // the advantages are complete from here on
+    grid_dependency_release();
+#pragma unroll
+    for (int i = 0; i < kWarpIters; ++i) {
+        int seq;
+        int64_t end;
+        if (nle < 32) { // the owner of this lane's first token: `own` plus the boundaries at or below it
+            int c = 0;
+            for (int j = 0; j < nle; ++j) c += (int64_t)__shfl_sync(kFull, bound, j) <= k0[i];
+            seq = own + c;
+            end = (int64_t)__shfl_sync(kFull, bound, c);
+        } else {        // more than 32 sequences in 512 tokens: every lane searches
+            seq = owner_sequence(a.cu, a.n_seq, min(k0[i], last), own);
+            end = (int64_t)__ldg(a.cu + seq + 1);
+        }
+        if (cnt[i] == 0)
+            continue;
+        float A = __ldg(a.adv + seq);
+        float coef = (float)(-(double)A * invN);
+        uint32_t w[8], rr[8];
+        uint2 chi = make_uint2(0u, 0u);
+        if (cnt[i] == 8 && k0[i] + 8 <= end) {
+            if (A >= 0.0f) coeffs8<KL, EXTRA, 0, true>(sn[i], so[i], sr[KL ? i : 0], mk[i], A, coef, nkl, hi, lo, w, rr, chi);
+            else coeffs8<KL, EXTRA, 0, false>(sn[i], so[i], sr[KL ? i : 0], mk[i], A, coef, nkl, hi, lo, w, rr, chi);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                if (e < cnt[i] && k0[i] + e >= end) { // into the next non-empty sequence
+                    while (seq + 1 < a.n_seq && k0[i] + e >= end) {
+                        ++seq;
+                        end = (int64_t)__ldg(a.cu + seq + 1);
+                    }
+                    A = __ldg(a.adv + seq);
+                    coef = (float)(-(double)A * invN);
+                }
+                const bool m = (((e < 4 ? mk[i].x : mk[i].y) >> (8 * (e & 3))) & 0xFFu) != 0;
+                float r;
+                bool c;
+                w[e] = __float_as_uint(omega_scalar<0>(__uint_as_float(sn[i][e]), __uint_as_float(so[i][e]),
+                                                       KL ? __uint_as_float(sr[KL ? i : 0][e]) : 0.0f, m, KL, A, coef, nkl, hi,
+                                                       lo, r, c));
+                rr[e] = __float_as_uint(r);
+                if (e < 4) chi.x |= (uint32_t)c << (8 * e);
+                else chi.y |= (uint32_t)c << (8 * (e - 4));
+            }
+        }
+        if (cnt[i] == 8) {
+            st_global_256(a.omega + k0[i], w);
+            if (EXTRA) {
+                if (a.ratio) st_global_256(a.ratio + k0[i], rr);
+                if (a.clip_mask) *reinterpret_cast<uint2 *>(a.clip_mask + k0[i]) = chi;
+            }
+        } else {
+            for (int e = 0; e < cnt[i]; ++e) {
+                a.omega[k0[i] + e] = __uint_as_float(w[e]);
+                if (EXTRA) {
+                    if (a.ratio) a.ratio[k0[i] + e] = __uint_as_float(rr[e]);
+                    if (a.clip_mask) a.clip_mask[k0[i] + e] = (uint8_t)(((e < 4 ? chi.x : chi.y) >> (8 * (e & 3))) & 1u);
                 }
             }
         }
@@ -1421,8 +1547,8 @@ extern "C" int hilore_grpo_coeffs_packed(const float *rewards, int64_t n_resp_to
         return HILORE_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t n_groups = (resp_offset + n_seq + G - 1) / G - resp_offset / G;
-    packed_advantage_kernel<<<(unsigned)((n_groups + 3) / 4), 128, 0, st>>>(rewards, resp_offset, n_seq, G, adv_eps, adv_out);
-    if (cudaGetLastError() != cudaSuccess)
+    if (launch_dependent(packed_advantage_kernel, dim3((unsigned)((n_groups + 3) / 4)), dim3(128), 0, st, rewards, resp_offset,
+                         n_seq, (int)G, adv_eps, adv_out) != cudaSuccess || cudaGetLastError() != cudaSuccess)
         return HILORE_CUDA;
     if (n_tok == 0)
         return HILORE_OK;
@@ -1442,8 +1568,19 @@ extern "C" int hilore_grpo_coeffs_packed(const float *rewards, int64_t n_resp_to
     a.omega = omega;
     a.ratio = ratio;
     a.clip_mask = clip_mask;
-    const int64_t tiles = (n_tok + kCoeffTile - 1) / kCoeffTile;
     const bool kl = beta != 0.0f, extra = (ratio != nullptr) || (clip_mask != nullptr);
+    if (aligned(logp_new, 32) && aligned(logp_old, 32) && aligned(a.logp_ref, 32) && aligned(omega, 32) && aligned(ratio, 32) &&
+        aligned(mask, 8) && aligned(clip_mask, 8)) { // the warp-tile kernel, as a programmatic dependent of the advantages
+        const int64_t wtiles = (n_tok + kWarpTile - 1) / kWarpTile;
+        const int64_t grid = (wtiles + kCoeffThreads / 32 - 1) / (kCoeffThreads / 32);
+        void (*wk)(PackedArgs, uint32_t) =
+            kl ? (extra ? grpo_coeffs_packed_warp_kernel<true, true> : grpo_coeffs_packed_warp_kernel<true, false>)
+               : (extra ? grpo_coeffs_packed_warp_kernel<false, true> : grpo_coeffs_packed_warp_kernel<false, false>);
+        if (launch_dependent(wk, dim3((unsigned)grid), dim3(kCoeffThreads), 0, st, a, (uint32_t)wtiles) != cudaSuccess)
+            return HILORE_CUDA;
+        return cudaGetLastError() == cudaSuccess ? HILORE_OK : HILORE_CUDA;
+    }
+    const int64_t tiles = (n_tok + kCoeffTile - 1) / kCoeffTile;
     void (*kernel)(PackedArgs) = kl ? (extra ? grpo_coeffs_packed_kernel<true, true> : grpo_coeffs_packed_kernel<true, false>)
                                     : (extra ? grpo_coeffs_packed_kernel<false, true> : grpo_coeffs_packed_kernel<false, false>);
     kernel<<<(unsigned)tiles, kCoeffThreads, 0, st>>>(a);

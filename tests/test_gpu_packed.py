@@ -88,6 +88,53 @@ def test_packed_microbatch_slice_device_normaliser_and_empty_sequences():
     check(ro, pk2, got, 1e-3, N)
 
 
+@pytest.mark.parametrize("beta", [0.0, 1e-3])
+@pytest.mark.parametrize("tail", [0, 3, 13])
+def test_packed_tiny_empty_and_long_sequences_in_one_microbatch(beta, tail):
+    """The warp-tile kernel's cases in one microbatch: runs of sequences of 0-13 tokens (more than 32 sequence starts
+    inside one 512-token tile, boundaries inside a lane's eight tokens, empty sequences), long sequences that span
+    several tiles, and a token count that is not a multiple of eight (outputs between canaries).  Against the oracle,
+    and bit for bit against the generic kernel, which the same call takes when a tensor is only 16-byte aligned."""
+    rng = np.random.default_rng(77 + tail)
+    G_ = 8
+    lens = np.concatenate([rng.choice([0, 0, 1, 2, 3, 5, 8, 13], 400), rng.integers(600, 1500, 9), rng.choice([0, 1, 7, 9], 150),
+                           rng.integers(600, 1500, 8), rng.choice([0, 2, 8, 16], 57)])
+    rng.shuffle(lens[:409])
+    lens[-1] += (tail - int(lens.sum())) % 8                  # token count = tail (mod 8)
+    n_seq = len(lens)
+    assert n_seq % G_ == 0
+    ro = synth.rollout(5, n_seq // G_, G_, 4, rewards="bernoulli", equal_group_fraction=0.2)
+    n_tok = int(lens.sum())
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    lp = rng.normal(-1.5, 0.5, n_tok).astype(np.float32)
+    pk = synth.PackedRollout(cu, np.arange(n_seq), lp, (lp + rng.normal(0, 0.12, n_tok)).astype(np.float32),
+                             (lp + rng.normal(0, 0.1, n_tok)).astype(np.float32), (rng.random(n_tok) < 0.8).astype(np.uint8),
+                             np.zeros(n_tok, np.int64))
+    N = int(pk.mask.sum())
+    got = packed_gpu(ro, pk, beta=beta, N=N)
+    check(ro, pk, got, beta, N)
+
+    def shifted(a, dtype):                                  # the same values at an address that is 16 mod 32 (masks: 4 mod 8)
+        t = torch.zeros(len(a) + 64, dtype=dtype, device="cuda")
+        off = 4 + (-(t.data_ptr() // 4) % 8 if dtype == torch.float32 else -t.data_ptr() % 8)
+        v = t[off:off + len(a)]
+        v.copy_(torch.from_numpy(np.ascontiguousarray(a)))
+        return v
+    ln, lo, lr, mk = shifted(pk.logp_new, torch.float32), shifted(pk.logp_old, torch.float32), shifted(pk.logp_ref, torch.float32), \
+        shifted(pk.mask, torch.uint8)
+    assert ln.data_ptr() % 32 == 16 and mk.data_ptr() % 8 == 4
+    adv = torch.zeros(n_seq, device="cuda")
+    omega, ratio = shifted(np.zeros(n_tok, np.float32), torch.float32), shifted(np.zeros(n_tok, np.float32), torch.float32)
+    chi = shifted(np.zeros(n_tok, np.uint8), torch.uint8)
+    api.hilore_grpo_coeffs_packed(G.dev(ro.rewards), ro.n_resp, ro.G, 0, n_seq, dev_i32(cu), n_tok, ln, lo, lr if beta else None,
+                                  mk, N, None, 0.2, beta, 1e-6, adv, omega, ratio, chi)
+    torch.cuda.synchronize()
+    assert np.array_equal(adv.cpu().numpy().view(np.uint32), got[0].view(np.uint32))
+    assert np.array_equal(omega.cpu().numpy().view(np.uint32), got[1].view(np.uint32))
+    assert np.array_equal(ratio.cpu().numpy().view(np.uint32), got[2].view(np.uint32))
+    assert np.array_equal(chi.cpu().numpy(), got[3])
+
+
 def test_packed_argument_errors():
     z = torch.zeros(16, device="cuda")
     zi = torch.zeros(4, dtype=torch.int32, device="cuda")
