@@ -52,10 +52,10 @@ NOMINAL_HBM_GBS = 8000.0
 # unit [16384, 18944] (five times the L2; summarised under profiles/; traffic grows in proportion to the
 # elements processed, every element being read once and written once).  Reads match the algorithmic reads; a
 # few percent of the written bytes are still dirty in L2 when such a single-unit kernel ends.
-DRAM_PER_ALGORITHMIC = {"compress": (620.847104 + 295.178240) / 950.6,   # codes + scales + token RMS
-                        "encode": (620.838144 + 289.419520) / 950.5,     # codes + scales
-                        "stats": (620.886528 + 3.636736) / 620.8,        # token RMS only
-                        "recover": (330.112768 + 562.481664) / 950.5}
+DRAM_PER_ALGORITHMIC = {"compress": (620.847616 + 296.770048) / 950.6,   # codes + scales + token RMS
+                        "encode": (620.838400 + 288.768000) / 950.5,     # codes + scales
+                        "stats": (620.841728 + 3.612672) / 620.8,        # token RMS only
+                        "recover": (329.943552 + 562.304512) / 950.5}
 
 
 # ---------------------------------------------------------------- accounting (bytes the method must move)
