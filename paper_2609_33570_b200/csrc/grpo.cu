@@ -766,20 +766,24 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
     __shared__ float s_A[FUSED ? kFusedRows : 1], s_coef[FUSED ? kFusedRows : 1];
     int64_t row_lo = 0;
     float f_kl = 0.0f, f_hi = 0.0f, f_lo = 0.0f;
+    bool pre = false; // FUSED: this thread's slots of the CTA's only piece are in registers already
+    uint32_t pre_m = 0;
+    float4 pre_sn = make_float4(0.0f, 0.0f, 0.0f, 0.0f), pre_so = pre_sn, pre_sr = pre_sn;
+    float4 pre_av[FUSED ? kExpUnits : 1];
     if (FUSED) { // the per-response scalars of the responses this CTA's slots belong to
         // This form runs at microbatch size, where the kernel is a chain of dependent memory latencies: ask for the
         // first piece's token data, the units' magnitudes and the plan inputs now, so that they arrive while the
         // group statistics (rewards -> fp64 sums -> shuffles) are worked out.
         {
             const int64_t k = (int64_t)tile * a.steps * kExpTile + (int64_t)tid * 4;
-            if (k < a.n_tok) {
+            if (k < a.n_tok && !(VEC && a.steps == 1)) { // (the one-piece form loads them into registers below)
                 prefetch_l2(a.f.logp_new + k);
                 prefetch_l2(a.f.logp_old + k);
                 if (a.f.logp_ref) prefetch_l2(a.f.logp_ref + k);
                 prefetch_l2(a.mask + k);
                 for (int j = 0; j < nu; ++j) prefetch_l2(a.row_rms + (int64_t)(u0 + j) * a.rms_ld + k);
             }
-            if (a.done != nullptr && a.plan.avail != nullptr && tid < nu) {
+            if ((a.done != nullptr || a.cluster) && a.plan.avail != nullptr && tid < nu) {
                 prefetch_l2(a.plan.kappa + u0 + tid);
                 prefetch_l2(a.plan.ebar + u0 + tid);
                 prefetch_l2(a.plan.avail + u0 + tid);
@@ -792,6 +796,22 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
         const int nrows = (int)((slot_hi - 1) / a.T - row_lo) + 1;
         const long long N = a.f.N_norm_dev ? *a.f.N_norm_dev : (long long)a.f.N_norm;
         const double invN = N > 0 ? 1.0 / (double)N : 0.0;
+        f_kl = (float)((double)a.f.beta * invN);
+        // One piece per CTA (the microbatch form): its token data and the units' magnitudes are loaded into
+        // registers now, so that only arithmetic is left once the statistics are known.
+        if (VEC && a.steps == 1) {
+            const int64_t k = slot_lo + (int64_t)tid * 4;
+            if (k < a.n_tok) {
+                pre = true;
+                pre_m = *reinterpret_cast<const unsigned int *>(a.mask + k);
+                pre_sn = *reinterpret_cast<const float4 *>(a.f.logp_new + k);
+                pre_so = *reinterpret_cast<const float4 *>(a.f.logp_old + k);
+                if (f_kl != 0.0f) pre_sr = *reinterpret_cast<const float4 *>(a.f.logp_ref + k);
+#pragma unroll
+                for (int j = 0; j < kExpUnits; ++j)
+                    if (j < nu) pre_av[j] = *reinterpret_cast<const float4 *>(a.row_rms + (int64_t)(u0 + j) * a.rms_ld + k);
+            }
+        }
         for (int r = wid; r < nrows; r += kExpThreads / 32) {
             const float A = group_advantage(a.f.rewards, a.f.resp_offset + row_lo + r, a.f.G, a.f.adv_eps, lane);
             if (lane == 0) {
@@ -799,7 +819,6 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
                 s_coef[r] = (float)(-(double)A * invN);
             }
         }
-        f_kl = (float)((double)a.f.beta * invN);
         f_hi = 1.0f + a.f.clip_eps;
         f_lo = 1.0f - a.f.clip_eps;
         __syncthreads();
@@ -872,13 +891,15 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
 #pragma unroll
             for (int i = 0; i < 4; ++i) slot[i] = k + i;
             if (k < a.n_tok) { // n_tok % 4 == 0: a group is valid as a whole
-                const uint32_t m = *reinterpret_cast<const unsigned int *>(a.mask + k);
+                const uint32_t m = (FUSED && pre) ? pre_m : *reinterpret_cast<const unsigned int *>(a.mask + k);
                 float wv[4];
                 if (FUSED) { // T % 4 == 0: the four slots belong to one response
-                    const float4 sn = *reinterpret_cast<const float4 *>(a.f.logp_new + k);
-                    const float4 so = *reinterpret_cast<const float4 *>(a.f.logp_old + k);
-                    float4 sr = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    if (f_kl != 0.0f) sr = *reinterpret_cast<const float4 *>(a.f.logp_ref + k);
+                    float4 sn = pre_sn, so = pre_so, sr = pre_sr;
+                    if (!pre) {
+                        sn = *reinterpret_cast<const float4 *>(a.f.logp_new + k);
+                        so = *reinterpret_cast<const float4 *>(a.f.logp_old + k);
+                        if (f_kl != 0.0f) sr = *reinterpret_cast<const float4 *>(a.f.logp_ref + k);
+                    }
                     const int ri = (int)(k / a.T - row_lo);
                     const float A = s_A[ri], coef = s_coef[ri];
                     wv[0] = fused_omega(sn.x, so.x, sr.x, (m & 0xFFu) != 0, A, coef, f_kl, f_hi, f_lo);
@@ -941,7 +962,7 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
                 float av[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                 if (VEC) {
                     if (slot[0] < a.n_tok) {
-                        const float4 t = *reinterpret_cast<const float4 *>(ar + slot[0]);
+                        const float4 t = (FUSED && pre) ? pre_av[FUSED ? j : 0] : *reinterpret_cast<const float4 *>(ar + slot[0]);
                         av[0] = t.x; av[1] = t.y; av[2] = t.z; av[3] = t.w;
                     }
                 } else {
