@@ -675,6 +675,7 @@ __global__ void __launch_bounds__(kCoeffThreads, 6) grpo_coeffs_packed_warp_kern
 constexpr int kExpThreads = 256;
 constexpr int kExpTile = kExpThreads * 4; // slots per CTA
 constexpr int kExpUnits = 8;              // units per CTA (omega and mask are read once for all of them)
+constexpr int kMaxClusterTiles = 16;      // CTAs (tiles of tokens) of a unit group in the cluster form
 
 // One warp adds the per-tile partials of unit u in a fixed order and applies the closed form
 //   E_u = (S2_u + eps * S3) / (S1_u / |T_b| + eps),  S1 = sum a, S2 = sum |omega| a, S3 = sum |omega|.
@@ -761,6 +762,10 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
     const int tile = blockIdx.x;
     const int u0 = blockIdx.y * kExpUnits, nu = min(kExpUnits, a.U - u0);
     __shared__ double sm[kExpThreads / 32][2 * (kExpUnits + 1)];
+    namespace cg = cooperative_groups;
+    cg::cluster_group cl = cg::this_cluster();
+    if (a.cluster)
+        cl.barrier_arrive(); // first phase of the cluster barrier: once all have arrived, every CTA of the cluster runs
     grid_dependency_wait();
     grid_dependency_release(); // the final reduction may become resident; it waits for this grid to complete
     __shared__ float s_A[FUSED ? kFusedRows : 1], s_coef[FUSED ? kFusedRows : 1];
@@ -986,14 +991,16 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
         if (lane == 0) sm[wid][q] = (double)v;
     }
     __syncthreads();
-    __shared__ double s_part[2 * (kExpUnits + 1)]; // this CTA's partial sums, for the cluster form
+    // cluster form: the partial sums of the cluster's CTAs, tile by tile, in the shared memory of its first CTA
+    __shared__ double s_all[kMaxClusterTiles][2 * (kExpUnits + 1)];
+    if (a.cluster)
+        cl.barrier_wait(); // (long since complete) the first CTA's shared memory may be written now
     if (tid < 2 * (kExpUnits + 1)) {
         double t = 0.0;
         for (int w = 0; w < kExpThreads / 32; ++w) t += sm[w][tid];
         const int j = tid >> 1, which = tid & 1;
-        s_part[tid] = t;
         if (a.cluster) {
-            // the sums stay in shared memory
+            cl.map_shared_rank(&s_all[0][0], 0)[cl.block_rank() * (2 * (kExpUnits + 1)) + tid] = t;
         } else if (j < kExpUnits) {
             if (j < nu) a.part[((int64_t)(u0 + j) * a.ntiles + tile) * 2 + which] = t;
         } else if (a.done != nullptr) { // single-launch form: every unit group keeps its own copy of the token sums
@@ -1004,21 +1011,22 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
     }
     if (a.cluster) {
         // Cluster form of the single launch (microbatch sizes): the CTAs of a unit group -- one per tile of tokens --
-        // are one thread-block cluster.  After the cluster barrier the first CTA reads every CTA's partial sums from
-        // its shared memory (distributed shared memory), lane t taking tile t as the final kernel does, so the
-        // results are those of the other forms bit for bit; no partial sum goes through global memory, nothing is
-        // counted, nothing needs clearing.  A second barrier keeps the other CTAs' shared memory alive until then.
-        namespace cg = cooperative_groups;
-        cg::cluster_group cl = cg::this_cluster();
-        cl.sync();
-        if (cl.block_rank() == 0 && wid < nu) {
+        // are one thread-block cluster.  Every CTA has written its partial sums into the first CTA's shared memory
+        // (distributed shared memory) and arrives at the cluster barrier (release); the first CTA waits for all
+        // (acquire) and goes on alone, lane t taking tile t as the final kernel does, so the results are those of
+        // the other forms bit for bit.  No partial sum goes through global memory, nothing is counted, nothing needs
+        // clearing, and the other CTAs are gone as soon as they have arrived: nobody reads their shared memory.
+        cl.barrier_arrive();
+        if (cl.block_rank() != 0)
+            return;
+        cl.barrier_wait();
+        if (wid < nu) {
             double s1 = 0.0, s2 = 0.0, s3 = 0.0, cnt = 0.0;
             if (lane < (int)gridDim.x) {
-                const double *remote = cl.map_shared_rank(s_part, lane);
-                s1 = remote[2 * wid];
-                s2 = remote[2 * wid + 1];
-                s3 = remote[2 * kExpUnits];
-                cnt = remote[2 * kExpUnits + 1];
+                s1 = s_all[lane][2 * wid];
+                s2 = s_all[lane][2 * wid + 1];
+                s3 = s_all[lane][2 * kExpUnits];
+                cnt = s_all[lane][2 * kExpUnits + 1];
             }
             double s3_all;
             const float E = exposure_from_lane_sums(s1, s2, s3, cnt, a.eps_alpha, &s3_all);
@@ -1029,7 +1037,6 @@ __global__ void __launch_bounds__(kExpThreads) exposure_partial_kernel(const __g
                 if (a.plan.avail) decide_unit(a.plan, u, &E);
             }
         }
-        cl.sync();
         return;
     }
     if (a.done == nullptr)
@@ -1333,7 +1340,7 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     // Microbatch sizes: one thread-block cluster per unit group (up to 16 CTAs, one per tile), reduction through the
     // cluster's shared memory; no counters, no memset.  Tile counts that are not a cluster size the device schedules
     // (or a device that refuses the launch) take the counter form below.
-    if (single_launch && a.ntiles >= 1 && a.ntiles <= 16 && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
+    if (single_launch && a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
                          aligned(mask, 4) && aligned(row_rms, 16);
         void (*kernel)(ExpArgs) = nullptr;
