@@ -26,10 +26,10 @@ struct CodecWork {
     int phase;                // HILORE_PHASE_* for table mode; CodecOp for single mode
     const uint8_t *avail;     // q_u
     const uint8_t *action;    // a_u
-    int64_t seg_bytes;        // size of the window all CTAs sweep together
+    int64_t seg_bytes;        // scale of the windows all CTAs sweep together (see plan_unit)
     uint64_t share_m;         // 2^32 = share_m * grid + share_rem
     uint32_t share_rem;
-    uint32_t rot_step;        // rotation of the CTA index per window (0 for a single unit)
+    uint32_t rot_step;        // rotation of the CTA index per window (0 for grids of one or two CTAs)
 };
 
 __device__ __forceinline__ int unit_op(const CodecWork &wk, int u)
