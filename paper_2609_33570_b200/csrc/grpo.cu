@@ -1340,7 +1340,8 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     // Microbatch sizes: one thread-block cluster per unit group (up to 16 CTAs, one per tile), reduction through the
     // cluster's shared memory; no counters, no memset.  Tile counts that are not a cluster size the device schedules
     // (or a device that refuses the launch) take the counter form below.
-    if (single_launch && a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
+    // Every caller of the reduction takes this form at these sizes (it needs no workspace and no second launch).
+    if (a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
                          aligned(mask, 4) && aligned(row_rms, 16);
         void (*kernel)(ExpArgs) = nullptr;
