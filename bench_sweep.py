@@ -393,7 +393,7 @@ def main():
     ap.add_argument("--no-coeffs", action="store_true")
     ap.add_argument("--no-rms", action="store_true", help="compress without the fused token RMS")
     ap.add_argument("--plan-table", action="store_true", help="only the 7B-shaped table under several candidate plans")
-    ap.add_argument("--case", choices=["codec", "coeffs", "coeffs-packed", "exposure", "scores"], help="run one small single-kernel case and exit")
+    ap.add_argument("--case", choices=["codec", "coeffs", "coeffs-packed", "exposure", "scores", "allocate", "relerr", "diagnostics"], help="run one small single-kernel case and exit")
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--fmt", type=int, default=api.FMT_E4M3FN_BLK)
     ap.add_argument("--units", type=int, default=2)
@@ -413,6 +413,12 @@ def main():
         score_refresh_case(a.reps)
     elif a.case == "coeffs-packed":
         print(json.dumps(coeffs_packed_point(a.log2_slots, a.reps)))
+    elif a.case == "allocate":
+        print(json.dumps(allocate_point(a.U, a.reps)))
+    elif a.case == "relerr":
+        print(json.dumps(relerr_point(a.rows, a.cols, a.fmt, a.reps)))
+    elif a.case == "diagnostics":
+        print(json.dumps(diagnostics_point(a.log2_slots, a.reps)))
     if a.case:
         print("done")
         return

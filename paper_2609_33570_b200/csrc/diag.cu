@@ -45,11 +45,13 @@ __device__ __forceinline__ void abs_bits4(const DiagArgs &a, int64_t k, bool vec
     }
 }
 
-// One shared-memory increment per distinct bin among the active lanes of a warp.
-__device__ __forceinline__ void hist_add(unsigned int *sh, uint32_t bin)
+// One shared-memory increment per distinct bin among the lanes of a warp that have a value (`active`); every lane of
+// the warp calls this.  (Plain atomics measure 10 % slower on B200 for the top digits of |omega|, which take a dozen
+// values per warp; electing the bins one by one with a shuffle and a ballot each, twice slower.)
+__device__ __forceinline__ void hist_add(unsigned int *sh, uint32_t bin, bool active)
 {
-    const unsigned peers = __match_any_sync(__activemask(), bin);
-    if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31))
+    const unsigned peers = __match_any_sync(0xFFFFFFFFu, active ? bin : 0xFFFFFFFFu);
+    if (active && (int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31))
         atomicAdd(&sh[bin], (unsigned)__popc(peers));
 }
 
@@ -73,35 +75,46 @@ __global__ void __launch_bounds__(kDiagThreads) diag_count_kernel(const __grid_c
     unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
     double sum = 0.0;
     const int64_t quads = (a.n + 3) / 4, stride = (int64_t)gridDim.x * kDiagThreads;
-    for (int64_t q = (int64_t)blockIdx.x * kDiagThreads + threadIdx.x; q < quads; q += stride) {
-        const int64_t k = 4 * q;
-        uint32_t b[4];
-        int cnt;
-        abs_bits4(a, k, vec, b, cnt);
-        float r[4];
-        if (vec && cnt == 4) {
-            const uint4 w = ld_global_128_stream(a.ratio + k);
-            r[0] = __uint_as_float(w.x), r[1] = __uint_as_float(w.y), r[2] = __uint_as_float(w.z), r[3] = __uint_as_float(w.w);
-        } else {
-            for (int j = 0; j < 4; ++j) r[j] = j < cnt ? a.ratio[k + j] : 0.0f;
+    // whole warps stay in the loop together (hist_add is a warp-wide call); a lane beyond the end has no value
+    for (int64_t q0 = (int64_t)blockIdx.x * kDiagThreads + (threadIdx.x & ~31); q0 < quads; q0 += stride) {
+        const int64_t q = q0 + (threadIdx.x & 31);
+        const bool in = q < quads;
+        const int64_t k = in ? 4 * q : 0;
+        uint32_t b[4] = {0, 0, 0, 0};
+        int cnt = 0;
+        float r[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        uint32_t mword = 0; // the four mask bytes, one per slot
+        if (in) {
+            abs_bits4(a, k, vec, b, cnt);
+            if (vec && cnt == 4) {
+                const uint4 w = ld_global_128_stream(a.ratio + k);
+                r[0] = __uint_as_float(w.x), r[1] = __uint_as_float(w.y), r[2] = __uint_as_float(w.z), r[3] = __uint_as_float(w.w);
+                mword = *reinterpret_cast<const uint32_t *>(a.mask + k);
+            } else {
+                for (int j = 0; j < cnt; ++j) {
+                    r[j] = a.ratio[k + j];
+                    mword |= (uint32_t)(a.mask[k + j] != 0) << (8 * j);
+                }
+            }
         }
         int64_t row = k / a.T, col = k - row * a.T;
-        float A = a.adv[row];
+        float A = in ? a.adv[row] : 0.0f;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            if (j < cnt) {
-                const bool m = a.mask[k + j] != 0;
+            const bool act = j < cnt;
+            if (act) {
+                const bool m = ((mword >> (8 * j)) & 0xFFu) != 0;
                 if (!m) ++c0;
                 else if (A == 0.0f) ++c1;
                 else if ((A > 0.0f && r[j] > hi) || (A < 0.0f && r[j] < lo)) ++c2;
                 if (b[j] == 0) ++c3;
                 sum += (double)__uint_as_float(b[j]);
-                hist_add(sh, b[j] >> 20);
                 if (++col == a.T && k + j + 1 < a.n) {
                     col = 0;
                     A = a.adv[++row];
                 }
             }
+            hist_add(sh, b[j] >> 20, act);
         }
     }
     atomicAdd(&sc[0], (unsigned long long)c0);
