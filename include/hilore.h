@@ -238,6 +238,11 @@ size_t hilore_omega_diagnostics_workspace_bytes(void);
  *   workspace     scratch of at least hilore_workspace_bytes(U, n_rows*T) bytes, 16-byte aligned; its
  *                 contents are overwritten (HILORE_WORKSPACE if too small).  Partial sums are kept in fp64
  *                 in fixed slots and added in a fixed order: the result is run-to-run deterministic.
+ *   Launches: at 1, 2, 4, 8 or 16 tiles of 1024 tokens the call is ONE launch (the CTAs of a group of eight units
+ *   are a thread-block cluster and add their sums through its shared memory; the workspace is not touched); other
+ *   sizes take a second, small launch that adds the partial sums of the workspace.  Same bits either way.  With
+ *   HILORE_DISABLE_CLUSTER_LAUNCH set in the environment (to anything but "0") no call of this library launches
+ *   thread-block clusters.
  */
 int hilore_unit_exposure(const float *omega, const uint8_t *mask, int64_t n_rows, int64_t T,
                          const float *row_rms, int32_t U, int64_t rms_ld, int32_t row_shift, float eps_alpha,

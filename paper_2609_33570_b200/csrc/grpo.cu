@@ -5,6 +5,8 @@
 
 #include <cooperative_groups.h>
 
+#include <cstdlib>
+
 namespace hilore {
 
 // ------------------------------------------------------------------ N = sum of the update mask
@@ -1341,7 +1343,11 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     // cluster's shared memory; no counters, no memset.  Tile counts that are not a cluster size the device schedules
     // (or a device that refuses the launch) take the counter form below.
     // Every caller of the reduction takes this form at these sizes (it needs no workspace and no second launch).
-    if (a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
+    // HILORE_DISABLE_CLUSTER_LAUNCH in the environment (any value but "0") sends every call through the workspace
+    // forms instead: same bits, for comparing the forms and for tools that cannot follow cluster launches.
+    const char *no_cluster = std::getenv("HILORE_DISABLE_CLUSTER_LAUNCH");
+    const bool clusters_on = no_cluster == nullptr || no_cluster[0] == '\0' || (no_cluster[0] == '0' && no_cluster[1] == '\0');
+    if (clusters_on && a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
                          aligned(mask, 4) && aligned(row_rms, 16);
         void (*kernel)(ExpArgs) = nullptr;

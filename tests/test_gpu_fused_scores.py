@@ -95,7 +95,7 @@ def scores_plan(ro, rms, sl, shapes, kappa, ebar, tau, avail, beta=0.0, row_shif
     (3, 4, 52, 3, "uniform", 0.0, 1),          # short rows, shifted rows
     (16, 16, 2048, 9, "uniform", 0.0, 0),      # 2^19 slots: coefficient pass first, then reduction + plan in one launch
 ])
-def test_single_launch_refresh_equals_the_separate_calls_and_the_oracle(P, G_, T, U, lengths, beta, row_shift):
+def test_single_launch_refresh_equals_the_separate_calls_and_the_oracle(P, G_, T, U, lengths, beta, row_shift, monkeypatch):
     ro = synth.rollout(71, P, G_, T, lengths=lengths, min_len=2, rewards="uniform", mask_first_column=bool(row_shift))
     ro.logp_old[:] = ro.logp_new + np.random.default_rng(5).normal(0, 0.1, ro.logp_new.shape).astype(np.float32)
     sl = slice(0, ro.n_resp)
@@ -125,6 +125,13 @@ def test_single_launch_refresh_equals_the_separate_calls_and_the_oracle(P, G_, T
     # twice in a row on the same workspace: the finished-CTA counter is left clean
     again = scores_plan(ro, rms, sl, shapes, kappa, ebar, tau, avail, beta, row_shift, fmt)
     assert again[1].tobytes() == E.tobytes() and np.array_equal(again[4], act)
+    # without thread-block clusters (the counter form of the single launch; workspace forms of the separate calls)
+    monkeypatch.setenv("HILORE_DISABLE_CLUSTER_LAUNCH", "1")
+    plain = scores_plan(ro, rms, sl, shapes, kappa, ebar, tau, avail, beta, row_shift, fmt)
+    assert plain[0].tobytes() == omega.tobytes() and plain[1].tobytes() == E.tobytes() and plain[3].tobytes() == psi.tobytes()
+    assert np.array_equal(plain[4], act) and np.array_equal(plain[6], ret)
+    omega3, E3, sw3 = fused(ro, rms, sl, beta=beta, row_shift=row_shift)
+    assert omega3.tobytes() == omega.tobytes() and E3.tobytes() == E.tobytes() and sw3 == sw
 
 
 def test_single_launch_refresh_argument_errors():

@@ -352,3 +352,24 @@ def test_fast_and_generic_coefficient_paths_give_the_same_bits(beta):
     fast, generic = run(0), run(4)
     for a, b in zip(fast, generic):
         assert a.tobytes() == b.tobytes()
+
+
+@pytest.mark.parametrize("tiles", [1, 2, 3, 4, 7, 8, 15, 16, 17, 33])
+def test_exposure_forms_give_the_same_bits_at_every_tile_count(tiles, monkeypatch):
+    """1, 2, 4, 8 and 16 tiles of 1024 tokens take the one-launch form (a thread-block cluster per group of eight units),
+    the other counts the workspace and a second kernel; with HILORE_DISABLE_CLUSTER_LAUNCH set every count does.  The
+    exposure scores are the oracle's to 1e-5 and the same bits in both forms; U = 11: a full and a partial unit group;
+    the last tile is ragged."""
+    T = 256
+    n_rows = 4 * tiles - 1
+    rng = np.random.default_rng(tiles)
+    omega = (rng.normal(0, 1e-5, (n_rows, T)) * (rng.random((n_rows, T)) < 0.7)).astype(np.float32)
+    mask = (rng.random((n_rows, T)) < 0.8).astype(np.uint8)
+    omega *= mask
+    rms = (rng.random((11, n_rows * T), dtype=np.float32) + np.float32(0.25))
+    E, sw = G.unit_exposure(omega, mask, rms)
+    oE, osw = oracle.unit_exposure(omega, mask, rms)
+    assert G.rel_err(E, oE).max() <= RTOL and abs(sw - osw) <= RTOL * osw
+    monkeypatch.setenv("HILORE_DISABLE_CLUSTER_LAUNCH", "1")
+    E2, sw2 = G.unit_exposure(omega, mask, rms)
+    assert E2.tobytes() == E.tobytes() and sw2 == sw
