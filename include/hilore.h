@@ -136,7 +136,7 @@ int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G
  * Eqs. "update-coefficient", "mlp-weighted-exposure", "token-weighted-risk", "available-recovery-actions").  The CTAs of
  * a group of eight units -- one per tile of 1024 tokens -- add their partial sums in the fixed order of the two-kernel
  * form and one of them takes the plan decisions of the group's units, so omega, exposure, psi, action_io, recompute and
- * retained_bytes are bit for bit those of the separate calls.  At microbatch size (1, 2, 4, 8 or 16 tiles) the CTAs of a
+ * retained_bytes are bit for bit those of the separate calls.  At microbatch size (up to 16 tiles of 1024 tokens; the cluster is the next power of two) the CTAs of a
  * group are one thread-block cluster and exchange the sums through its distributed shared memory; otherwise through
  * the workspace, the CTA that finishes last (a counter per group, cleared by a memset inside the call) doing the
  * rest.  Between forward and backward of a microbatch this is one launch instead of four.
@@ -238,9 +238,9 @@ size_t hilore_omega_diagnostics_workspace_bytes(void);
  *   workspace     scratch of at least hilore_workspace_bytes(U, n_rows*T) bytes, 16-byte aligned; its
  *                 contents are overwritten (HILORE_WORKSPACE if too small).  Partial sums are kept in fp64
  *                 in fixed slots and added in a fixed order: the result is run-to-run deterministic.
- *   Launches: at 1, 2, 4, 8 or 16 tiles of 1024 tokens the call is ONE launch (the CTAs of a group of eight units
- *   are a thread-block cluster and add their sums through its shared memory; the workspace is not touched); other
- *   sizes take a second, small launch that adds the partial sums of the workspace.  Same bits either way.  With
+ *   Launches: up to 16 tiles of 1024 tokens the call is ONE launch (the CTAs of a group of eight units are a
+ *   thread-block cluster and add their sums through its shared memory; the workspace is not touched); larger
+ *   microbatches take a second, small launch that adds the partial sums of the workspace.  Same bits either way.  With
  *   HILORE_DISABLE_CLUSTER_LAUNCH set in the environment (to anything but "0") no call of this library launches
  *   thread-block clusters.
  */

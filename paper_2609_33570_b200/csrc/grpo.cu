@@ -1339,15 +1339,18 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
     a.eps_alpha = eps_alpha;
     a.exposure = exposure;
     a.sum_abs_omega = sum_abs_omega;
-    // Microbatch sizes: one thread-block cluster per unit group (up to 16 CTAs, one per tile), reduction through the
-    // cluster's shared memory; no counters, no memset.  Tile counts that are not a cluster size the device schedules
-    // (or a device that refuses the launch) take the counter form below.
+    // Microbatch sizes (up to 16 tiles): one thread-block cluster per unit group, one CTA per tile, reduction through
+    // the cluster's shared memory; no counters, no memset.  More tiles (or a device that refuses the launch) take the
+    // forms below.
     // Every caller of the reduction takes this form at these sizes (it needs no workspace and no second launch).
     // HILORE_DISABLE_CLUSTER_LAUNCH in the environment (any value but "0") sends every call through the workspace
     // forms instead: same bits, for comparing the forms and for tools that cannot follow cluster launches.
     const char *no_cluster = std::getenv("HILORE_DISABLE_CLUSTER_LAUNCH");
     const bool clusters_on = no_cluster == nullptr || no_cluster[0] == '\0' || (no_cluster[0] == '0' && no_cluster[1] == '\0');
-    if (clusters_on && a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && (a.ntiles & (a.ntiles - 1)) == 0 && steps == 1) {
+    // A tile count that is not a power of two takes the next one: the CTAs beyond the last tile add zeros.
+    int csize = 1;
+    while (csize < a.ntiles) csize *= 2;
+    if (clusters_on && a.ntiles >= 1 && a.ntiles <= kMaxClusterTiles && steps == 1) {
         const bool vec = row_shift == 0 && (n_tok % 4 == 0) && (rms_ld % 4 == 0) && aligned(omega, 16) &&
                          aligned(mask, 4) && aligned(row_rms, 16);
         void (*kernel)(ExpArgs) = nullptr;
@@ -1358,16 +1361,16 @@ static int launch_exposure(const float *omega, const uint8_t *mask, int64_t n_ro
         } else {
             kernel = vec ? exposure_partial_kernel<true, false> : exposure_partial_kernel<false, false>;
         }
-        if (cluster_launch_ok(kernel, a.ntiles)) {
+        if (cluster_launch_ok(kernel, csize)) {
             a.cluster = 1;
             if (plan) a.plan = *plan;
             cudaLaunchConfig_t cfg{};
-            cfg.gridDim = dim3((unsigned)a.ntiles, (unsigned)groups);
+            cfg.gridDim = dim3((unsigned)csize, (unsigned)groups);
             cfg.blockDim = dim3(kExpThreads);
             cfg.stream = st;
             cudaLaunchAttribute attr[2];
             attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = (unsigned)a.ntiles;
+            attr[0].val.clusterDim.x = (unsigned)csize;
             attr[0].val.clusterDim.y = 1;
             attr[0].val.clusterDim.z = 1;
             attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
