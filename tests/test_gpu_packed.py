@@ -135,6 +135,29 @@ def test_packed_tiny_empty_and_long_sequences_in_one_microbatch(beta, tail):
     assert np.array_equal(chi.cpu().numpy(), got[3])
 
 
+def test_packed_coefficients_of_a_whole_rollout_batch_of_2p24_tokens():
+    """The largest point of the sweep on this layout: 2^24 + 5 tokens in about 8200 sequences of 1-3 K tokens (with a
+    few empty ones and a run of very short ones), every token against the oracle, with the K3 term."""
+    rng = np.random.default_rng(2024)
+    G_, target = 8, (1 << 24) + 5
+    lens = rng.integers(1024, 3073, 9000)
+    lens[100:140] = rng.choice([0, 1, 2, 5], 40)
+    lens = lens[: int(np.searchsorted(np.cumsum(lens), target)) + 1]
+    lens[-1] -= int(lens.sum()) - target
+    lens = np.concatenate([lens, np.zeros((-len(lens)) % G_, np.int64)])       # empty sequences fill the last group
+    n_seq, n_tok = len(lens), int(lens.sum())
+    assert n_tok == target and lens.min() >= 0
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    ro = synth.rollout(9, n_seq // G_, G_, 4, rewards="bernoulli", equal_group_fraction=0.1)
+    lp = rng.normal(-1.5, 0.5, n_tok).astype(np.float32)
+    pk = synth.PackedRollout(cu, np.arange(n_seq), lp, (lp + rng.normal(0, 0.1, n_tok)).astype(np.float32),
+                             (lp + rng.normal(0, 0.08, n_tok)).astype(np.float32), (rng.random(n_tok) < 0.75).astype(np.uint8),
+                             np.zeros(n_tok, np.int64))
+    N = int(pk.mask.sum())
+    got = packed_gpu(ro, pk, beta=1e-3, N=N)
+    check(ro, pk, got, 1e-3, N)
+
+
 def test_packed_argument_errors():
     z = torch.zeros(16, device="cuda")
     zi = torch.zeros(4, dtype=torch.int32, device="cuda")
