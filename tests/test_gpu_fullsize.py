@@ -2,7 +2,7 @@
 
 The microbatch the benchmark times as its headline (7B-shaped, 24 GB) and two microbatches of the 1.5B-shaped step are
 compared with the oracle WHOLE (its C calls spread over row ranges on the host cores).  Where a test samples instead
-(the 4 GiB unit, the demotion run): a row's codes, scales, token RMS and reconstruction depend on that row only, so
+(the demotion run, the mixed table): a row's codes, scales, token RMS and reconstruction depend on that row only, so
 the oracle can check any sample of rows.  Inputs are drawn on the device with the same recipe as the host generators
 (N(0,1), 1 % of the channels x20)."""
 import numpy as np
