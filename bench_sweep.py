@@ -5,9 +5,9 @@ coefficient kernel over 2^16 ... 2^24 slots at G = 16.  Each point is timed with
 calls that rotate through a pool of distinct buffers larger than L2, so the numbers are HBM numbers.
 Prints one JSON line per point.  `bench.py` imports the point functions for the per-config legs of its line.
 
-`--case codec|coeffs|exposure` runs one small single-kernel case a few times and exits: inputs larger than
-L2, well under a few GB on the device, a handful of launches -- the cases the profiler captures under
-`profiles/` were taken on.
+`--case codec|coeffs|coeffs-packed|exposure|scores|allocate|relerr|diagnostics` runs one small single-kernel case
+a few times and exits: inputs larger than L2 where the kernel streams, well under a few GB on the device, a handful
+of launches -- the cases the profiler captures under `profiles/` were taken on.
 """
 from __future__ import annotations
 
