@@ -123,8 +123,15 @@ def _ptr(t):
     return t.data_ptr()
 
 
+# the current stream's handle without building a Stream object (3.2 us -> 1.2 us per call where torch has these)
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+_raw_device = getattr(torch._C, "_cuda_getDevice", None)
+
+
 def _stream(stream):
     if stream is None:
+        if _raw_stream is not None and _raw_device is not None:
+            return _raw_stream(_raw_device())
         return torch.cuda.current_stream().cuda_stream
     return stream if isinstance(stream, int) else stream.cuda_stream
 
