@@ -117,7 +117,7 @@ int hilore_grpo_coeffs(const float *rewards, int64_t n_resp_total, int32_t G, in
 /*
  * hilore_grpo_coeffs followed by hilore_unit_exposure as ONE sweep (Algorithm 1, "coefficients" and "exposure"
  * lines; Eqs. "update-coefficient", "mlp-weighted-exposure"): the coefficients are computed inside the exposure
- * reduction instead of being written and read back, which saves a launch and the round trip of omega when the
+ * reduction instead of being written and read back, which saves launches and the round trip of omega when the
  * microbatch is small enough for the call to be launch-bound (n_rows * T <= 2^18 slots and at most 62 responses
  * per 1024 slots; other shapes run the two passes in turn inside this call).  Results are bit for bit those of
  * the two calls: omega [n_rows, T] (REQUIRED here, it is written either way), exposure [U], sum_abs_omega (opt).
@@ -136,10 +136,11 @@ int hilore_coeffs_exposure(const float *rewards, int64_t n_resp_total, int32_t G
  * Eqs. "update-coefficient", "mlp-weighted-exposure", "token-weighted-risk", "available-recovery-actions").  The CTAs of
  * a group of eight units -- one per tile of 1024 tokens -- add their partial sums in the fixed order of the two-kernel
  * form and one of them takes the plan decisions of the group's units, so omega, exposure, psi, action_io, recompute and
- * retained_bytes are bit for bit those of the separate calls.  At microbatch size (up to 16 tiles of 1024 tokens; the cluster is the next power of two) the CTAs of a
- * group are one thread-block cluster and exchange the sums through its distributed shared memory; otherwise through
- * the workspace, the CTA that finishes last (a counter per group, cleared by a memset inside the call) doing the
- * rest.  Between forward and backward of a microbatch this is one launch instead of four.
+ * retained_bytes are bit for bit those of the separate calls.  At microbatch size (up to 16 tiles of 1024 tokens;
+ * the cluster is the next power of two) the CTAs of a group are one thread-block cluster and hand the sums to its
+ * first CTA through distributed shared memory; otherwise through the workspace, the CTA that finishes last (a
+ * counter per group, cleared by a memset inside the call) doing the rest.  Between forward and backward of a
+ * microbatch this is one launch instead of four.
  *   Arguments as in hilore_coeffs_exposure (omega REQUIRED, U > 0, n_rows * T > 0) and in the DECIDE phase of
  *   hilore_plan_apply (units_dev, kappa, ebar, avail, action_io REQUIRED; psi, recompute, retained_bytes opt; the
  *   unit table is only read for rows, cols and fmt, on the device).
