@@ -75,7 +75,7 @@ struct UnitPlan {
 };
 
 // `per_row`: a per-row result (token RMS) is wanted.
-__device__ __forceinline__ UnitPlan plan_unit(const CodecWork &wk, const hilore_unit &u, bool per_row)
+__device__ __forceinline__ UnitPlan plan_unit(const CodecWork &wk, const hilore_unit &u, bool per_row, bool recover)
 {
     UnitPlan p;
     int64_t item_bytes = u.cols * 2;
@@ -101,9 +101,15 @@ __device__ __forceinline__ UnitPlan plan_unit(const CodecWork &wk, const hilore_
     // (a single unit shared by rows is cut from seg_bytes on: units of 128-141 MiB compress 3-5 % faster in two
     // windows when they are alone in the launch, and 3 % slower when they are part of a table; below seg_bytes two
     // windows lose up to 7 %)
-    const int64_t uncut = (wk.units == nullptr && !p.flat) ? wk.seg_bytes : wk.seg_bytes + wk.seg_bytes / 2;
+    // A unit alone in its launch and shared by 16 KB pieces likewise, in windows of half of seg_bytes (recover of the
+    // scaled formats at 128 MiB / 512 MiB / 4 GiB 5.51 -> 5.62, 6.08 -> 6.20, 6.38 -> 6.45 TB/s, compress without
+    // token RMS 2-4 % faster); the recover pass of the unscaled format keeps the larger windows (2 % faster with them
+    // at 128 MiB).
+    const bool alone = wk.units == nullptr;
+    const bool small_pieces = alone && p.flat && !(recover && u.fmt == HILORE_FMT_E4M3FN_RAW);
+    const int64_t uncut = (alone && (!p.flat || small_pieces)) ? wk.seg_bytes : wk.seg_bytes + wk.seg_bytes / 2;
     if (unit_bytes >= uncut) {
-        const int64_t window = p.flat ? wk.seg_bytes : max(wk.seg_bytes * 2 / 3, 9 * nC * item_bytes / 2);
+        const int64_t window = small_pieces ? wk.seg_bytes / 2 : p.flat ? wk.seg_bytes : max(wk.seg_bytes * 2 / 3, 9 * nC * item_bytes / 2);
         const int64_t nseg = max((int64_t)1, (unit_bytes + window / 2) / window);
         p.seg_items = (p.items + nseg - 1) / nseg;
     }
@@ -137,7 +143,7 @@ __device__ __forceinline__ void stage_units(const CodecWork &wk, bool recover, U
             if (op == OP_COMPRESS && wk.units && wk.phase == HILORE_PHASE_ENCODE)
                 u.row_rms = nullptr; // token magnitudes were collected at capture time
             st.u[t] = u;
-            st.plan[t] = plan_unit(wk, u, !recover && u.row_rms != nullptr);
+            st.plan[t] = plan_unit(wk, u, !recover && u.row_rms != nullptr, recover);
         }
         st.op[t] = op;
     }
