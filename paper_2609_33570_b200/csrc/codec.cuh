@@ -101,13 +101,13 @@ __device__ __forceinline__ UnitPlan plan_unit(const CodecWork &wk, const hilore_
     // (a single unit shared by rows is cut from seg_bytes on: units of 128-141 MiB compress 3-5 % faster in two
     // windows when they are alone in the launch, and 3 % slower when they are part of a table; below seg_bytes two
     // windows lose up to 7 %)
-    // A unit alone in its launch and shared by 16 KB pieces likewise, in windows of half of seg_bytes (recover of the
-    // scaled formats at 128 MiB / 512 MiB / 4 GiB 5.51 -> 5.62, 6.08 -> 6.20, 6.38 -> 6.45 TB/s, compress without
-    // token RMS 2-4 % faster); the recover pass of the unscaled format keeps the larger windows (2 % faster with them
-    // at 128 MiB).
+    // A unit alone in its launch and shared by 16 KB pieces is cut from 1.5 x seg_bytes on like the others, but into
+    // windows of half of seg_bytes (E4M3FN + scales: recover at 0.5 / 1 / 4 GiB 6.11 -> 6.21, 6.23 -> 6.31, 6.39 -> 6.44
+    // TB/s, compress without token RMS 2-4 % faster); the recover pass of the unscaled and the INT8 format keeps the
+    // larger windows (1-3 % faster with them).
     const bool alone = wk.units == nullptr;
-    const bool small_pieces = alone && p.flat && !(recover && u.fmt == HILORE_FMT_E4M3FN_RAW);
-    const int64_t uncut = (alone && (!p.flat || small_pieces)) ? wk.seg_bytes : wk.seg_bytes + wk.seg_bytes / 2;
+    const bool small_pieces = alone && p.flat && !(recover && u.fmt != HILORE_FMT_E4M3FN_BLK);
+    const int64_t uncut = (alone && !p.flat) ? wk.seg_bytes : wk.seg_bytes + wk.seg_bytes / 2;
     if (unit_bytes >= uncut) {
         const int64_t window = small_pieces ? wk.seg_bytes / 2 : p.flat ? wk.seg_bytes : max(wk.seg_bytes * 2 / 3, 9 * nC * item_bytes / 2);
         const int64_t nseg = max((int64_t)1, (unit_bytes + window / 2) / window);
